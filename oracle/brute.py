@@ -1,0 +1,79 @@
+"""Dense brute force for tiny inputs: a second, differently written statement of the same
+definitions, used only to cross-check the C oracle.  Test infrastructure only.
+
+* ``plan_tokens`` / ``plan_pages``: Algorithm 1's budgeted selection written with Python sets
+  (the C oracle uses a flag array and an insertion sort; this uses ``sorted`` with a key).
+* ``dense_attention``: gathers the whole context of a sequence into dense [L, d] matrices through
+  the block table, builds an explicit 0/1 visibility vector per query row, sets the logits of
+  invisible tokens to -inf and applies a plain softmax (Section 3.2: the proposal path sees the
+  plan's pages, the verifier sees everything up to the row's own position).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def _bf16_to_f64(bits):
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def plan_tokens(L, spans, budget, n_sink, n_recent):
+    """spans: list of (start, length, score).  Returns (set of selected tokens, over_budget)."""
+    chosen = set(range(0, min(n_sink, L))) | set(range(max(0, L - n_recent), L)) | {L - 1}
+    if len(chosen) > budget:
+        return chosen, True
+    clipped = []
+    for idx, (start, length, score) in enumerate(spans):
+        lo, hi = max(0, int(start)), min(L, int(start) + int(length))
+        if hi > lo:
+            clipped.append((-float(np.float32(score)), lo, idx, hi))
+    for _, lo, _, hi in sorted(clipped):
+        fresh = set(range(lo, hi)) - chosen
+        if len(chosen) + len(fresh) <= budget:
+            chosen |= fresh
+    return chosen, False
+
+
+def plan_pages(L, spans, budget, n_sink, n_recent, page_size=16, force_full=False):
+    """Returns (ascending logical page list, number of selected tokens, over_budget)."""
+    if force_full:
+        return list(range((L + page_size - 1) // page_size)), L, False
+    tokens, over = plan_tokens(L, spans, budget, n_sink, n_recent)
+    return sorted({t // page_size for t in tokens}), len(tokens), over
+
+
+def dense_attention(q_bits, pool_bits, bt_pages, L, visible_pages, n_q, scale=None):
+    """One sequence.  q_bits [n_q, Hq, d]; pool_bits [pages, 2, Hkv, P, d]; bt_pages: the
+    sequence's block table (logical -> physical); visible_pages: iterable of logical pages the
+    rows may see (all pages for verification).  Row j sits at position L - n_q + j.
+    Returns (out [n_q, Hq, d], lse [n_q, Hq], weights [n_q, Hq, L])."""
+    q = _bf16_to_f64(q_bits)
+    pool = _bf16_to_f64(pool_bits)
+    _, _, Hkv, P, d = pool.shape
+    Hq = q.shape[1]
+    G = Hq // Hkv
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    n_pages = (L + P - 1) // P
+    phys = np.asarray(bt_pages[:n_pages], dtype=np.int64)
+    # dense [L, Hkv, d]
+    K = pool[phys, 0].transpose(0, 2, 1, 3).reshape(n_pages * P, Hkv, d)[:L]
+    V = pool[phys, 1].transpose(0, 2, 1, 3).reshape(n_pages * P, Hkv, d)[:L]
+    page_vis = np.zeros(n_pages, dtype=bool)
+    page_vis[list(visible_pages)] = True
+    tok_vis = np.repeat(page_vis, P)[:L]
+    out = np.zeros((n_q, Hq, d))
+    lse = np.zeros((n_q, Hq))
+    weights = np.zeros((n_q, Hq, L))
+    for j in range(n_q):
+        pos = L - n_q + j
+        vis = tok_vis & (np.arange(L) <= pos)
+        for h in range(Hq):
+            z = scale * (K[:, h // G, :] @ q[j, h])
+            z = np.where(vis, z, -np.inf)
+            m = z.max()
+            e = np.exp(z - m)
+            weights[j, h] = e / e.sum()
+            out[j, h] = weights[j, h] @ V[:, h // G, :]
+            lse[j, h] = m + np.log(e.sum())
+    return out, lse, weights

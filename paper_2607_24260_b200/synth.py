@@ -1,0 +1,356 @@
+"""Seeded synthetic inputs shaped like the paper's 4K-128K long-context QA sweep.
+
+This module only *draws inputs*: context lengths, ranked evidence spans, budgets, block tables
+and bf16 Q/K/V values.  It contains none of the method's arithmetic (no plan compilation, no
+attention), so both the CUDA library's tests/benchmark and the CPU oracle's tests can share it
+without sharing any of the computation under test.
+
+The paper's experiments (Section 5.1, "Context-length control") keep a query's core evidence
+fixed and let low-priority context grow from 4K to 128K tokens, so the retained-KV ratio falls
+from about 40 % to 5.5 % (Table 2).  The generators below reproduce that structure with seeded
+random spans: a small set of ranked evidence spans over a long context, an always-kept sink prefix
+and recent suffix, and a token budget.  They stand in for the SPIQA-based prompts, which are not
+available offline.
+
+All host randomness comes from ``numpy.random.Generator(Philox(key=...))`` keyed by
+``(seed, workload, purpose)`` so that every draw is reproducible and independent of call order.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+import zlib
+from typing import Optional, Sequence
+
+import numpy as np
+
+NUM_Q_HEADS = 32
+NUM_KV_HEADS = 8
+HEAD_DIM = 128
+PAGE_SIZE = 16
+
+
+# ----------------------------------------------------------------------------- rng / bf16 helpers
+def rng_for(seed: int, *tags) -> np.random.Generator:
+    """Philox generator keyed by (seed, tags...) - tags are hashed with crc32 (stable)."""
+    h = zlib.crc32(repr(tags).encode("utf-8"))
+    return np.random.Generator(np.random.Philox(key=[np.uint64(seed), np.uint64(h)]))
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even float32 -> bfloat16 bit patterns (uint16). NaN stays NaN."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32)
+    rounding = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    out = ((u + rounding) >> np.uint32(16)).astype(np.uint16)
+    nan = np.isnan(x)
+    if nan.any():
+        out = np.where(nan, np.uint16(0x7FC0), out)
+    return out
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    b = np.ascontiguousarray(b, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
+    return bf16_bits_to_f32(b).astype(np.float64)
+
+
+def normal_bf16(shape, std: float, rng: np.random.Generator) -> np.ndarray:
+    """N(0, std^2) samples rounded to bf16, returned as uint16 bit patterns."""
+    return f32_to_bf16_bits(rng.standard_normal(shape, dtype=np.float32) * np.float32(std))
+
+
+# ----------------------------------------------------------------------------------- the workload
+@dataclasses.dataclass
+class Workload:
+    """Everything the three entry points take, except the KV values themselves.
+
+    Arrays are host numpy arrays with the dtypes of the C ABI (int32 / float32 / uint8).
+    """
+    name: str
+    layers: int
+    ctx_len: np.ndarray            # [B] tokens in the KV cache (verification rows included)
+    n_q: np.ndarray                # [B] verification rows per sequence
+    span_indptr: np.ndarray        # [B+1]
+    span_start: np.ndarray         # [n_spans] token index of the span's first token
+    span_len: np.ndarray           # [n_spans]
+    span_score: np.ndarray         # [n_spans] float32 priority (higher = more relevant)
+    budget_tokens: np.ndarray      # [B]
+    n_sink: np.ndarray             # [B]
+    n_recent: np.ndarray           # [B]
+    force_full: np.ndarray         # [B] uint8, 1 = take the full-context fallback path
+    bt_indptr: np.ndarray          # [B+1] CSR block table: logical page -> physical page
+    bt_pages: np.ndarray           # [sum pages]
+    num_pool_pages: int
+    s_max: float = 1.0
+    num_q_heads: int = NUM_Q_HEADS
+    num_kv_heads: int = NUM_KV_HEADS
+    head_dim: int = HEAD_DIM
+    page_size: int = PAGE_SIZE
+    note: str = ""
+
+    @property
+    def batch(self) -> int:
+        return int(self.ctx_len.shape[0])
+
+    @property
+    def q_indptr(self) -> np.ndarray:
+        out = np.zeros(self.batch + 1, dtype=np.int32)
+        np.cumsum(self.n_q, out=out[1:])
+        return out
+
+    @property
+    def page_bytes(self) -> int:
+        """Bytes of one KV page of one layer (K and V, all KV heads)."""
+        return 2 * self.num_kv_heads * self.page_size * self.head_dim * 2
+
+    @property
+    def pool_elems_per_layer(self) -> int:
+        return self.num_pool_pages * 2 * self.num_kv_heads * self.page_size * self.head_dim
+
+    def pages_of(self, b: int) -> int:
+        return int(self.bt_indptr[b + 1] - self.bt_indptr[b])
+
+
+def _pages(L: int, page: int = PAGE_SIZE) -> int:
+    return (int(L) + page - 1) // page
+
+
+def block_tables(ctx_len: Sequence[int], mode: str, seed: int, tag: str,
+                 page_size: int = PAGE_SIZE, spare_pages: int = 0):
+    """CSR block tables for a batch.
+
+    ``sequential``: sequence b owns a contiguous run of physical pages, in order.
+    ``shuffled``  : the physical pages of the whole batch are one random permutation of the
+                    shared pool (what a long-running paged allocator converges to).
+    ``spare_pages`` extra never-referenced pages are appended to the pool.
+    """
+    n = np.array([_pages(L, page_size) for L in ctx_len], dtype=np.int64)
+    indptr = np.zeros(len(n) + 1, dtype=np.int32)
+    np.cumsum(n, out=indptr[1:])
+    total = int(indptr[-1])
+    pool = total + int(spare_pages)
+    if mode == "sequential":
+        pages = np.arange(total, dtype=np.int32)
+    elif mode == "shuffled":
+        pages = rng_for(seed, tag, "block_table").permutation(pool)[:total].astype(np.int32)
+    else:
+        raise ValueError(f"unknown block-table mode {mode!r}")
+    return indptr, pages, pool
+
+
+def _pack_spans(per_seq):
+    indptr = np.zeros(len(per_seq) + 1, dtype=np.int32)
+    np.cumsum([len(s[0]) for s in per_seq], out=indptr[1:])
+    cat = lambda i, dt: (np.concatenate([np.asarray(s[i], dtype=dt) for s in per_seq])
+                         if per_seq else np.zeros(0, dtype=dt))
+    return indptr, cat(0, np.int32), cat(1, np.int32), cat(2, np.float32)
+
+
+def _uniform_spans(rng, L, n_spans, span_tokens):
+    """n_spans spans of span_tokens tokens with uniform starts; scores are a seeded
+    permutation of the ranks n_spans..1 (distinct, so the ranking has no ties)."""
+    starts = rng.integers(0, max(1, L - span_tokens + 1), size=n_spans)
+    scores = rng.permutation(n_spans).astype(np.float32) + 1.0
+    return starts, np.full(n_spans, span_tokens), scores
+
+
+def _zipf_chunk_spans(rng, L, chunk_tokens, zipf_s, len_lo, len_hi):
+    """One candidate span per chunk_tokens-token chunk; the chunk of rank r (1 = best) scores
+    r**-zipf_s, ranks assigned by a seeded permutation.  With len_lo == len_hi == chunk_tokens the
+    span is the chunk itself; otherwise its length is uniform in [len_lo, len_hi], centred on the
+    chunk centre and clipped to [0, L) - unaligned and sometimes overlapping its neighbours."""
+    n_chunks = max(1, L // chunk_tokens)
+    ranks = rng.permutation(n_chunks) + 1
+    scores = (ranks.astype(np.float64) ** (-zipf_s)).astype(np.float32)
+    if len_lo == len_hi == chunk_tokens:
+        starts = np.arange(n_chunks) * chunk_tokens
+        lens = np.full(n_chunks, chunk_tokens)
+    else:
+        lens = rng.integers(len_lo, len_hi + 1, size=n_chunks)
+        centre = np.arange(n_chunks) * chunk_tokens + chunk_tokens // 2
+        starts = np.clip(centre - lens // 2, 0, None)
+        lens = np.minimum(lens, L - starts)
+    return starts, lens, scores
+
+
+def _finish(name, layers, ctx_len, n_q, spans, budget, sink, recent, force_full, bt_mode, seed,
+            note="", spare_pages=0, s_max=1.0) -> Workload:
+    B = len(ctx_len)
+    si, ss, sl, sc = _pack_spans(spans)
+    bi, bp, pool = block_tables(ctx_len, bt_mode, seed, name, spare_pages=spare_pages)
+    as_i32 = lambda v: np.ascontiguousarray(np.broadcast_to(np.asarray(v, dtype=np.int32), (B,)))
+    return Workload(
+        name=name, layers=layers, ctx_len=as_i32(ctx_len), n_q=as_i32(n_q),
+        span_indptr=si, span_start=ss, span_len=sl, span_score=sc,
+        budget_tokens=as_i32(budget), n_sink=as_i32(sink), n_recent=as_i32(recent),
+        force_full=np.ascontiguousarray(np.broadcast_to(
+            np.asarray(force_full, dtype=np.uint8), (B,))),
+        bt_indptr=bi, bt_pages=bp, num_pool_pages=pool, s_max=s_max, note=note)
+
+
+# ------------------------------------------------------------------- the five named configurations
+def config1(seed: int = 0, clip_budget: bool = False) -> Workload:
+    """Single sequence, single layer, 4096 tokens: 64 sink + 128 recent + 8 spans x 64 tokens.
+    The stated "about 11 %" does not match 704 tokens of 4096 (17 %), so the primary run leaves
+    the budget open (budget = L); ``clip_budget`` runs the 11 % budget (450 tokens) instead."""
+    L = 4096
+    rng = rng_for(seed, "c1", "spans")
+    spans = [_uniform_spans(rng, L, 8, 64)]
+    budget = int(0.11 * L) if clip_budget else L
+    return _finish("c1b" if clip_budget else "c1", 1, [L], 4, spans, budget, 64, 128, 0,
+                   "sequential", seed, note="B=1 L=4096 1 layer; verify k=4")
+
+
+def config2(seed: int = 0, batch: int = 8, L: int = 16384, layers: int = 32) -> Workload:
+    """Llama-3-8B attention shape, batch 8, 16K context, 10 % budget from 16 spans x 96 tokens."""
+    spans = [_uniform_spans(rng_for(seed, "c2", "spans", b), L, 16, 96) for b in range(batch)]
+    return _finish("c2", layers, [L] * batch, 4, spans, int(0.10 * L), 64, 256, 0,
+                   "sequential", seed, note=f"B={batch} L={L} {layers} layers; verify k=4")
+
+
+def config3(seed: int = 0, batch: int = 16, L: int = 32768, layers: int = 32,
+            bt_mode: str = "sequential") -> Workload:
+    """Batch 16, 32K context, Zipf(1.1)-ranked 256-token chunks turned into 128-512-token
+    spans, 8 % budget.  Sink/recent are unstated for this configuration: 64 + 256 as config 2."""
+    spans = [_zipf_chunk_spans(rng_for(seed, "c3", "spans", b), L, 256, 1.1, 128, 512)
+             for b in range(batch)]
+    return _finish("c3", layers, [L] * batch, 8, spans, int(0.08 * L), 64, 256, 0, bt_mode, seed,
+                   note=f"B={batch} L={L} {layers} layers; verify k=8")
+
+
+def config4(seed: int = 0, batch: int = 4, L: int = 131072, layers: int = 32,
+            bt_mode: str = "sequential") -> Workload:
+    """Batch 4, 128K context, 5.5 % budget from Zipf-ranked page-aligned 256-token chunks."""
+    spans = [_zipf_chunk_spans(rng_for(seed, "c4", "spans", b), L, 256, 1.1, 256, 256)
+             for b in range(batch)]
+    return _finish("c4", layers, [L] * batch, 4, spans, int(0.055 * L), 64, 512, 0, bt_mode, seed,
+                   note=f"B={batch} L={L} {layers} layers; verify k=4")
+
+
+def config5(seed: int = 0, batch: int = 32, layers: int = 16, lo: int = 4096,
+            hi: int = 131072) -> Workload:
+    """Mixed serving batch: log-uniform lengths, budgets uniform in 3-20 %, 10 % of the sequences
+    on the full-context fallback path, verify k in {4, 8}, ragged block tables over one shuffled
+    shared pool."""
+    rng = rng_for(seed, "c5", "shape")
+    ctx = np.rint(np.exp(rng.uniform(math.log(lo), math.log(hi), size=batch))).astype(np.int64)
+    frac = rng.uniform(0.03, 0.20, size=batch)
+    n_full = max(1, int(round(0.10 * batch)))
+    force = np.zeros(batch, dtype=np.uint8)
+    force[rng.choice(batch, size=n_full, replace=False)] = 1
+    n_q = rng.choice(np.array([4, 8]), size=batch)
+    spans = [_zipf_chunk_spans(rng_for(seed, "c5", "spans", b), int(ctx[b]), 256, 1.1, 128, 512)
+             for b in range(batch)]
+    budget = np.floor(frac * ctx).astype(np.int64)
+    recent = np.minimum(256, ctx // 8)
+    return _finish("c5", layers, ctx, n_q, spans, budget, 64, recent, force, "shuffled", seed,
+                   note=f"{batch} ragged seqs {lo}-{hi} tokens, {layers} layers; k in {{4,8}}")
+
+
+CONFIGS = {"c1": config1, "c1b": lambda seed=0: config1(seed, clip_budget=True),
+           "c2": config2, "c3": config3, "c4": config4, "c5": config5}
+
+
+def tiny_random(seed: int, batch: int = 3, max_len: int = 200, max_spans: int = 12,
+                page_size: int = PAGE_SIZE, bt_mode: str = "shuffled", spare_pages: int = 3,
+                adversarial: bool = True) -> Workload:
+    """Small random cases for brute-force comparison: overlapping spans, score ties, spans that
+    stick out of [0, L), empty spans, budgets around the mandatory size, occasional fallback."""
+    rng = rng_for(seed, "tiny")
+    ctx = rng.integers(1, max_len + 1, size=batch)
+    spans, budget, sink, recent, force, nq = [], [], [], [], [], []
+    for b in range(batch):
+        L = int(ctx[b])
+        n = int(rng.integers(0, max_spans + 1))
+        if adversarial:
+            starts = rng.integers(-8, L + 8, size=n)
+            lens = rng.integers(0, max(2, L // 2 + 2), size=n)
+            scores = rng.integers(0, 4, size=n).astype(np.float32) / 2.0      # many ties
+        else:
+            starts = rng.integers(0, L, size=n)
+            lens = rng.integers(1, max(2, L // 3 + 1), size=n)
+            scores = rng.random(n).astype(np.float32)
+        spans.append((starts, lens, scores))
+        budget.append(int(rng.integers(0, L + 8)))
+        sink.append(int(rng.integers(0, 10)))
+        recent.append(int(rng.integers(0, 24)))
+        force.append(int(rng.random() < 0.1))
+        nq.append(int(rng.integers(1, min(9, L) + 1)))
+    bi, bp, pool = block_tables(ctx, bt_mode, seed, "tiny", page_size, spare_pages)
+    si, ss, sl, sc = _pack_spans(spans)
+    i32 = lambda v: np.asarray(v, dtype=np.int32)
+    return Workload(name=f"tiny{seed}", layers=1, ctx_len=i32(ctx), n_q=i32(nq), span_indptr=si,
+                    span_start=ss, span_len=sl, span_score=sc, budget_tokens=i32(budget),
+                    n_sink=i32(sink), n_recent=i32(recent),
+                    force_full=np.asarray(force, dtype=np.uint8), bt_indptr=bi, bt_pages=bp,
+                    num_pool_pages=pool, page_size=page_size)
+
+
+# ------------------------------------------------------------------------------------ value draws
+def host_qkv(w: Workload, seed: int, layer: int = 0, kv_std: float = 0.5, q_std: float = 1.0,
+             q_rows: Optional[int] = None):
+    """Host-side bf16 bit patterns for one layer: ``pool[num_pool_pages, 2, Hkv, P, d]`` (HND,
+    K then V per page) with N(0, kv_std^2) values and ``q[q_rows, Hq, d]`` with N(0, q_std^2).
+    Only for cases small enough to generate on the CPU."""
+    rng = rng_for(seed, w.name, "kv", layer)
+    pool = normal_bf16((w.num_pool_pages, 2, w.num_kv_heads, w.page_size, w.head_dim), kv_std, rng)
+    rows = int(w.n_q.sum()) if q_rows is None else int(q_rows)
+    q = normal_bf16((rows, w.num_q_heads, w.head_dim), q_std, rng_for(seed, w.name, "q", layer))
+    return q, pool
+
+
+def device_fill_normal_(t, std: float, seed: int, chunk_elems: int = 1 << 27):
+    """Fill a (large) torch CUDA bf16 tensor in place with N(0, std^2) from a seeded device
+    generator, chunk by chunk so the fp32 staging buffer stays small."""
+    import torch
+    g = torch.Generator(device=t.device)
+    g.manual_seed(int(seed))
+    flat = t.view(-1)
+    n = flat.numel()
+    stage = torch.empty(min(n, chunk_elems), dtype=torch.float32, device=t.device)
+    for off in range(0, n, chunk_elems):
+        m = min(chunk_elems, n - off)
+        stage[:m].normal_(0.0, std, generator=g)
+        flat[off:off + m].copy_(stage[:m])
+    return t
+
+
+def plant_affinity_keys_(pool_layer, q_layer, w: Workload, phys_pages_per_seq, seed: int,
+                         layer: int, prob: float = 0.125, sigmas: float = 2.0,
+                         kv_std: float = 0.5, q_std: float = 1.0):
+    """Give a seeded subset of the keys inside the given (selected) pages a raw dot-product
+    affinity of +``sigmas`` standard deviations with one query head of their KV group:
+    ``k_t += (delta / |q_h|^2) q_h`` with ``delta = sigmas * sqrt(d) * q_std * kv_std`` (the
+    standard deviation of a raw q.k dot product), then round to bf16.  ``pool_layer`` is a torch
+    bf16 tensor [pages, 2, Hkv, P, d], ``q_layer`` a torch bf16 tensor [B, Hq, d] (one query row
+    per sequence), ``phys_pages_per_seq`` a list of int arrays.  In place; returns the count."""
+    import torch
+    G = w.num_q_heads // w.num_kv_heads
+    delta = sigmas * math.sqrt(w.head_dim) * q_std * kv_std
+    planted = 0
+    for b, pages in enumerate(phys_pages_per_seq):
+        pages = np.asarray(pages, dtype=np.int64)
+        if pages.size == 0:
+            continue
+        rng = rng_for(seed, w.name, "plant", layer, b)
+        shape = (pages.size, w.num_kv_heads, w.page_size)
+        hit = rng.random(shape) < prob
+        which = rng.integers(0, G, size=shape)
+        pi, gi, ti = np.nonzero(hit)
+        if pi.size == 0:
+            continue
+        dev = pool_layer.device
+        head = torch.as_tensor(gi * G + which[pi, gi, ti], device=dev)
+        qh = q_layer[b].float()[head]                                   # [n, d]
+        bump = qh * (delta / (qh * qh).sum(-1, keepdim=True).clamp_min(1e-6))
+        p_idx = torch.as_tensor(pages[pi], device=dev)
+        g_idx = torch.as_tensor(gi, device=dev)
+        t_idx = torch.as_tensor(ti, device=dev)
+        cur = pool_layer[p_idx, 0, g_idx, t_idx].float()
+        pool_layer[p_idx, 0, g_idx, t_idx] = (cur + bump).to(pool_layer.dtype)
+        planted += int(pi.size)
+    return planted
