@@ -1,0 +1,234 @@
+/*
+ * kap.h - C ABI of the B200 (sm_100a) library for the KAP / GraphSpec decode hot path:
+ * decode-time attention over the selected-KV view that a runtime access plan defines, and the
+ * full-context verification attention that guards it.
+ *
+ * The three operations come from the KAP paper (Section 2.1, Eq. 1: the runtime access plan
+ * A = (U, M, pos, rho_access, rho_verify); Section 3.1, Algorithm 1: the GraphSpec compiler;
+ * Section 3.2: the GraphSpec executor's two paths):
+ *
+ *   kap_compile_plan          Algorithm 1 from "token spans" onward: budgeted selection of ranked
+ *                             evidence spans (U), resolution to KV pages and physical pages through
+ *                             the block table (M), logical page indices kept (pos), fallback flags.
+ *   kap_selected_decode_attn  "Selected-KV proposal": one query row per sequence (q_prop = 1) at
+ *                             its full-sequence logical position, attending only to the plan's
+ *                             pages of the paged KV pool.
+ *   kap_verify_attn           "Full-context verification": n_q contiguous query rows per sequence
+ *                             over the whole block table, original logical positions, causal among
+ *                             the rows.
+ *
+ * Conventions
+ *   - Plain C, no exceptions, no aborts: every call returns a kap_status; kap_last_error() gives
+ *     a thread-local message for the last failure on the calling thread.
+ *   - Pointers are marked HOST or DEVICE.  The caller owns every buffer it passes; the library
+ *     owns only kap_workspace objects.
+ *   - The attention calls only enqueue kernels on the given CUDA stream and return (asynchronous,
+ *     no allocation, no synchronisation; they can be captured into a CUDA graph).  Problems a
+ *     kernel detects (a page index outside the pool, a bounded wait that ran out) set a status
+ *     word that kap_workspace_check() reads.
+ *   - KV pool layout of one layer ("HND"): bf16 pool[page][2][Hkv][P][d], index 0 = K, 1 = V, so the
+ *     K (or V) rows of one page and one KV head are P*d contiguous elements.  Supported shape:
+ *     d = 128, P = 16, Hq = G*Hkv with G in {1, 2, 4, 8, 16}; anything else is KAP_ERR_UNSUPPORTED.
+ *     The pool base address must be 16-byte aligned.
+ *   - Keys in the pool are already position-encoded at their logical index and queries arrive
+ *     encoded at theirs (the paper's logical-position preservation, Section 2.1); the kernels
+ *     apply no positional operation - positions only decide visibility.
+ */
+#ifndef KAP_H_
+#define KAP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KAP_OK = 0,
+    KAP_ERR_INVALID_ARG = 1,   /* malformed input; outputs untouched */
+    KAP_ERR_CAPACITY = 2,      /* result does not fit the caller's buffers / the workspace */
+    KAP_ERR_UNSUPPORTED = 3,   /* shape outside the supported set */
+    KAP_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed */
+    KAP_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out */
+    KAP_ERR_DEVICE_INDEX = 6   /* a kernel met an out-of-range page or list index */
+} kap_status;
+
+/* per-sequence plan flags (bit-or) written by kap_compile_plan */
+enum {
+    KAP_PLAN_FULL = 1,         /* identity plan: the sequence takes full-context access */
+    KAP_PLAN_OVER_BUDGET = 2,  /* the mandatory tokens alone exceed the budget; no span selected */
+    KAP_PLAN_S_HIGH = 4        /* retained ratio s (Eq. 4, in pages) > s_max: caller should fall back */
+};
+
+/*
+ * kap_compile_plan - Algorithm 1, steps SelectEvidenceUnderBudget, ResolveSelectedKVObjects,
+ * PreserveLogicalPositions, BuildBlockTable (Section 3.1).  HOST pointers in and out; runs on the
+ * calling thread; touches no GPU.  Runs once per request (the paper counts it inside TTFT).
+ *
+ * Per sequence b with L = ctx_len[b] tokens and n_pages = ceil(L / page_size):
+ *   1. mandatory tokens: the sink prefix [0, n_sink), the recent suffix [L - n_recent, L) and the
+ *      last token L-1.  They count toward the budget.  If they alone exceed budget_tokens[b] the
+ *      plan is the mandatory set and KAP_PLAN_OVER_BUDGET is set.
+ *   2. spans span_indptr[b] .. span_indptr[b+1]-1 are clipped to [0, L) (empty ones dropped) and
+ *      ranked by score descending, then clipped start ascending, then input index ascending.
+ *   3. first fit over whole spans: a span is taken iff the tokens it adds to the union fit the
+ *      remaining budget; otherwise it is skipped and the scan continues.  Spans are never cut.
+ *   4. a logical page is selected iff it holds a selected token; pages are emitted in ascending
+ *      logical order; plan_phys_pages[i] = bt_pages[bt_indptr[b] + plan_logical_pages[i]].
+ *   5. force_full[b] != 0 selects every page and sets KAP_PLAN_FULL (the fallback path, Section 3.2
+ *      "Runtime stability and fallback"); selected/total pages > s_max sets KAP_PLAN_S_HIGH.
+ *
+ * plan_indptr[batch+1], plan_flags[batch] and selected_tokens[batch] (may be NULL) are written;
+ * plan_logical_pages / plan_phys_pages receive plan_indptr[batch] entries and must hold
+ * plan_capacity entries.  plan_phys_pages may be NULL; it requires a block table otherwise.
+ * force_full and the block table may be NULL.
+ *
+ * Errors: KAP_ERR_INVALID_ARG for batch < 0, page_size <= 0, ctx_len <= 0, a negative budget /
+ * sink / recent / span length, a NaN score, a non-monotone span_indptr, a block table shorter than
+ * n_pages, a negative block-table entry, or a required pointer that is NULL; KAP_ERR_CAPACITY when
+ * the plan needs more than plan_capacity entries (the paper's "plan exceeds the compact workspace"
+ * fallback condition).  On any error no output is written.
+ */
+kap_status kap_compile_plan(
+    int32_t batch, int32_t page_size,
+    const int32_t* ctx_len,            /* HOST [batch] tokens in the KV cache incl. the current one */
+    const int32_t* span_indptr,        /* HOST [batch+1] */
+    const int32_t* span_start,         /* HOST [n_spans] first token of each span */
+    const int32_t* span_len,           /* HOST [n_spans] */
+    const float* span_score,           /* HOST [n_spans] priority, higher first */
+    const int32_t* budget_tokens,      /* HOST [batch] */
+    const int32_t* n_sink,             /* HOST [batch] */
+    const int32_t* n_recent,           /* HOST [batch] */
+    const uint8_t* force_full,         /* HOST [batch] or NULL */
+    float s_max,                       /* >= 1 disables the KAP_PLAN_S_HIGH test */
+    const int32_t* bt_indptr,          /* HOST [batch+1] CSR block table, or NULL */
+    const int32_t* bt_pages,           /* HOST logical page -> physical page */
+    int64_t plan_capacity,
+    int32_t* plan_indptr,              /* HOST out [batch+1] */
+    int32_t* plan_logical_pages,       /* HOST out, ascending per sequence */
+    int32_t* plan_phys_pages,          /* HOST out or NULL */
+    int32_t* plan_flags,               /* HOST out [batch] */
+    int32_t* selected_tokens);         /* HOST out [batch] or NULL: size of the token union */
+
+/*
+ * Workspace: the split-K work list of one launch shape and the buffers for the partial results
+ * (the paper's "reusable workspace" and stable metadata shapes, Section 3.2 "Runtime stability and
+ * fallback").  The paper has no counterpart for the split-K schedule itself; it is how this
+ * library spreads one sequence's page list over the GPU's SMs.
+ *
+ * kap_workspace_create allocates (cudaMalloc / cudaMallocHost) on `device`:
+ *   max_items          most work items (CTAs) one schedule may hold
+ *   max_rows_per_item  most query rows of one (sequence, KV head): n_q * (Hq / Hkv)
+ *   max_batch          most sequences
+ * kap_schedule (HOST arrays) splits every (sequence, KV head) page list of list_len[b] pages into
+ * near-equal contiguous chunks so that the chunks fill the GPU in whole waves, uploads the work
+ * list on `cuda_stream` (asynchronous copy from pinned memory owned by the workspace) and keeps
+ * it until the next kap_schedule.  The schedule depends only on the page counts, so one schedule
+ * serves every layer and every step whose list lengths and row counts are unchanged.
+ * A workspace serves one attention call at a time: use one for the proposal path and another for
+ * the verification path.  max_chunk_pages = 0 picks the default chunk cap.
+ * Errors: KAP_ERR_INVALID_ARG (NULL, batch < 0 or > max_batch, list_len <= 0, n_q < 1, bad head
+ * counts), KAP_ERR_CAPACITY (rows or items beyond what the workspace was created for),
+ * KAP_ERR_CUDA.
+ */
+typedef struct kap_workspace kap_workspace;
+
+kap_status kap_workspace_create(kap_workspace** ws, int32_t device, int32_t max_items,
+                                int32_t max_rows_per_item, int32_t max_batch);
+void kap_workspace_destroy(kap_workspace* ws);
+
+kap_status kap_schedule(
+    kap_workspace* ws, int32_t batch,
+    const int32_t* list_len,           /* HOST [batch] pages in each sequence's list */
+    const int32_t* n_q,                /* HOST [batch] query rows per sequence, NULL => 1 each */
+    int32_t num_q_heads, int32_t num_kv_heads,
+    int32_t max_chunk_pages,           /* cap on pages per work item, 0 => default */
+    void* cuda_stream);
+
+/* The schedule kap_schedule would build for `cta_slots` resident CTAs per wave, written to HOST
+ * arrays without touching a GPU (for inspection and tests).  items_out holds max_items rows of
+ * 8 int32: seq, kv_head, page_begin, page_end (relative to the sequence's list), group, partial
+ * slot, n_splits, n_q; longest chunks first.  Any output pointer may be NULL.  Like kap_schedule
+ * it has no counterpart in the paper.  Errors as kap_schedule, minus KAP_ERR_CUDA. */
+kap_status kap_schedule_host(
+    int32_t batch, const int32_t* list_len, const int32_t* n_q, int32_t num_q_heads,
+    int32_t num_kv_heads, int32_t cta_slots, int32_t max_chunk_pages, int32_t max_items,
+    int32_t* items_out, int32_t* n_items, int32_t* n_merge_groups, int32_t* max_chunk);
+
+/* what the last kap_schedule produced; any pointer may be NULL */
+kap_status kap_schedule_info(const kap_workspace* ws, int32_t* n_items, int32_t* n_merge_groups,
+                             int32_t* max_chunk_pages, int32_t* ctas_per_wave);
+
+/*
+ * kap_selected_decode_attn - Section 3.2 "Selected-KV proposal".  For sequence b and query head h
+ * (KV head g = h / G), with Vis(b) = the tokens t < ctx_len[b] of the plan's pages:
+ *     z_t = sm_scale * <q[b,h,:], K[g,t,:]>,   out[b,h,:] = sum_t softmax_t(z) V[g,t,:],
+ *     lse[b,h] = ln sum_t exp(z_t)            (natural log)
+ * computed as split-K flash decoding (bf16 tensor-core products, fp32 accumulation, base-2 online
+ * softmax) followed by a log-sum-exp merge of the splits.  One layer per call.
+ * plan_logical_pages == NULL means "logical page = position in the list" (identity plan).
+ * The plan arrays are the DEVICE copies of kap_compile_plan's outputs; `ws` must hold a schedule
+ * made from the same per-sequence list lengths with n_q = NULL.
+ * Errors: KAP_ERR_INVALID_ARG (NULL pointer, batch mismatch with the schedule, misaligned pool),
+ * KAP_ERR_UNSUPPORTED (shape), KAP_ERR_CUDA (launch failure).  Nothing is enqueued on error.
+ */
+kap_status kap_selected_decode_attn(
+    const void* q,                     /* DEVICE bf16 [batch, Hq, d] */
+    const void* kv_pool,               /* DEVICE bf16 [num_pool_pages][2][Hkv][P][d], this layer */
+    int64_t num_pool_pages,
+    const int32_t* plan_indptr,        /* DEVICE [batch+1] */
+    const int32_t* plan_phys_pages,    /* DEVICE [plan_indptr[batch]] */
+    const int32_t* plan_logical_pages, /* DEVICE same length, or NULL */
+    const int32_t* ctx_len,            /* DEVICE [batch] */
+    int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
+    float sm_scale,
+    void* out,                         /* DEVICE bf16 [batch, Hq, d] */
+    float* lse,                        /* DEVICE fp32 [batch, Hq] or NULL */
+    kap_workspace* ws, void* cuda_stream);
+
+/*
+ * kap_verify_attn - Section 3.2 "Full-context verification".  Sequence b has n_q = q_indptr[b+1] -
+ * q_indptr[b] query rows (the paper's q_verify = k + 1 window, or k rows); row j sits at logical
+ * position p_j = ctx_len[b] - n_q + j and sees every token t <= p_j of the full block table
+ * (ctx_len counts the rows' own tokens, whose K/V are already in the pool: the verifier advances
+ * the full KV state in the same pass).  Same formula, same kernels as the proposal path.
+ * bt_pages may list more pages than ceil(ctx_len / P) per sequence; only the first
+ * ceil(ctx_len / P) are read.  `ws` must hold a schedule made from list_len[b] = ceil(ctx_len[b]/P)
+ * and the same n_q.  Errors as kap_selected_decode_attn.
+ */
+kap_status kap_verify_attn(
+    const void* q,                     /* DEVICE bf16 [sum n_q, Hq, d], a sequence's rows contiguous */
+    const int32_t* q_indptr,           /* DEVICE [batch+1] */
+    const void* kv_pool, int64_t num_pool_pages,
+    const int32_t* bt_indptr,          /* DEVICE [batch+1] CSR full block table */
+    const int32_t* bt_pages,           /* DEVICE */
+    const int32_t* ctx_len,            /* DEVICE [batch] */
+    int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
+    float sm_scale,
+    void* out,                         /* DEVICE bf16 [sum n_q, Hq, d] */
+    float* lse,                        /* DEVICE fp32 [sum n_q, Hq] or NULL */
+    kap_workspace* ws, void* cuda_stream);
+
+/* Synchronises `cuda_stream` and returns the device status word of the workspace (KAP_OK,
+ * KAP_ERR_TIMEOUT or KAP_ERR_DEVICE_INDEX), clearing it. */
+kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);
+
+/* Tuning knobs of the attention launches, process-wide: `use_pdl` != 0 launches with programmatic
+ * stream serialisation (the next kernel's prologue overlaps the previous kernel's tail);
+ * `fused_merge` != 0 lets the last split of a (sequence, KV head) to finish merge the splits
+ * inside the split kernel instead of launching the separate merge pass.  Negative = keep. */
+kap_status kap_set_launch_options(int32_t use_pdl, int32_t fused_merge);
+
+/* Number of kernels this library has launched in this process (all threads). */
+int64_t kap_launch_count(void);
+
+/* Thread-local text for the last non-OK status returned on this thread ("" if none). */
+const char* kap_last_error(void);
+
+/* "kap-b200 <major>.<minor> sm_100a" */
+const char* kap_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KAP_H_ */

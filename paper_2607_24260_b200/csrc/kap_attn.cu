@@ -1,0 +1,810 @@
+// Split-K paged attention for sm_100a: the kernels behind kap_selected_decode_attn (Section 3.2,
+// "Selected-KV proposal") and kap_verify_attn (Section 3.2, "Full-context verification") of the
+// KAP paper, plus the log-sum-exp merge of the splits.
+//
+// One CTA = one work item = a contiguous slice of one sequence's page list for one KV head.
+//   * a producer warp (one elected lane) walks the slice's physical page ids and issues TMA tensor
+//     loads (cp.async.bulk.tensor, 128-byte swizzle) of each page's K and V rows for this KV head
+//     into a ring of shared-memory stages, completion tracked by mbarriers;
+//   * four consumer warps each own one 16-row tile of query rows (rows = n_q * G: the G query
+//     heads of the KV head's group times the n_q query tokens, so every K/V byte is read from HBM
+//     once and shared by all of them), compute S = Q K^T and O += P V with bf16 mma.sync tiles and
+//     fp32 accumulators, and keep a base-2 online softmax per row in registers;
+//   * the warps' states are combined through shared memory and the CTA writes either the final
+//     bf16 output (single split) or an un-normalised fp32 partial (m, l, O) for the merge pass.
+// The proposal path is the n_q = 1 case of the same kernel; the causal rule "row j sees tokens
+// t <= L - n_q + j" covers both paths.
+//
+// Every device-side wait is bounded: when a wait passes the CTA's deadline the kernel records
+// KAP_ERR_TIMEOUT in the workspace status word and runs to its end without spinning again.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "kap_internal.h"
+
+namespace kap {
+
+kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t* n_q,
+                          int32_t num_q_heads, int32_t num_kv_heads, int32_t cta_slots,
+                          int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
+                          std::vector<WorkItem>& items, std::vector<MergeGroup>& groups,
+                          int32_t* max_chunk_out, int32_t* row_tiles_out);
+
+// ------------------------------------------------------------------------------ kernel geometry
+constexpr int kConsumerWarps = 4;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;       // + the producer warp
+constexpr int kStagePages = 4;                            // pages per pipeline stage
+constexpr int kStages = 3;
+constexpr int kHalfTileBytes = kPageSize * 128;           // 16 tokens x 64 bf16 = 2048 B
+constexpr int kTileBytes = 2 * kHalfTileBytes;            // K (or V) of one page and head: 4096 B
+constexpr int kPageHeadBytes = 2 * kTileBytes;            // K + V: 8192 B
+constexpr int kStageBytes = kStagePages * kPageHeadBytes; // 32 KiB
+constexpr int kMaxChunk = 512;                            // page ids a CTA can hold
+constexpr int kScratchStride = kHeadDim + 8;              // floats per scratch row (bank spread)
+constexpr uint64_t kWaitBudgetNs = 2000000000ull;         // per-CTA deadline for all waits
+
+struct SmemTail {                                         // what follows the tile ring
+    int32_t phys[kMaxChunk];
+    int32_t logical[kMaxChunk];
+    unsigned long long full[kStages];
+    unsigned long long empty[kStages];
+    float m[kConsumerWarps][kRowTile];
+    float l[kConsumerWarps][kRowTile];
+    int32_t is_last;
+    int32_t timed_out;
+};
+constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(SmemTail) + 1024;  // + alignment slack
+
+static_assert(kConsumerWarps * kRowTile * kScratchStride * 4 <= kStages * kStageBytes,
+              "warp-combine scratch must fit in the tile ring");
+
+struct AttnParams {
+    const __nv_bfloat16* q;          // [rows, Hq, d]
+    const int32_t* q_indptr;         // [B+1] or null: sequence b owns row b
+    const int32_t* list_indptr;      // [B+1]
+    const int32_t* phys_pages;
+    const int32_t* logical_pages;    // or null: logical page = position in the list
+    const int32_t* ctx_len;          // [B]
+    const WorkItem* items;
+    const MergeGroup* groups;
+    float* part_o;                   // [slots][rows_cap][128]
+    float* part_ml;                  // [slots][rows_cap][2]
+    int32_t* counters;               // [groups] arrival counters (fused merge)
+    __nv_bfloat16* out;              // [rows, Hq, d]
+    float* lse;                      // [rows, Hq] or null
+    int32_t* status;
+    long long num_pool_pages;
+    int32_t Hq, Hkv, G, rows_cap;
+    int32_t fused_merge;
+    float scale_log2;                // sm_scale * log2(e)
+};
+
+// ------------------------------------------------------------------------------- PTX primitives
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: spins until the phase completes or the CTA's deadline passes.  After the deadline
+// every wait tries once and gives up, so the kernel always terminates.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t deadline,
+                                          volatile int32_t* timed_out) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*timed_out) return false;
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 255u) == 0 && global_ns() > deadline) { *timed_out = 1; return false; }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x,
+                                            int32_t y, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                        uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                          uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                         uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+        "{%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+__device__ __forceinline__ void consumer_sync() {           // the 128 consumer threads only
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+}
+
+// ------------------------------------------------------------------ merging partial softmax states
+// Combine `n` states (m_i in log2 units, l_i, O_i[4]) read through the accessors into one.
+// Used for warps inside a CTA and for the splits of a (sequence, KV head).
+struct Merged { float m, l; float4 o; };
+
+template <typename GetM, typename GetL, typename GetO>
+__device__ __forceinline__ Merged merge_states(int n, GetM get_m, GetL get_l, GetO get_o) {
+    float mx = -INFINITY;
+    for (int i = 0; i < n; ++i) mx = fmaxf(mx, get_m(i));
+    const float mu = (mx == -INFINITY) ? 0.f : mx;
+    Merged r; r.m = mx; r.l = 0.f; r.o = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < n; ++i) {
+        const float w = ex2(get_m(i) - mu);
+        const float4 o = get_o(i);
+        r.l = fmaf(w, get_l(i), r.l);
+        r.o.x = fmaf(w, o.x, r.o.x); r.o.y = fmaf(w, o.y, r.o.y);
+        r.o.z = fmaf(w, o.z, r.o.z); r.o.w = fmaf(w, o.w, r.o.w);
+    }
+    return r;
+}
+
+// normalise, round to bf16 and store 4 consecutive outputs; lse in natural log
+__device__ __forceinline__ void store_final(const AttnParams& p, int64_t q_row, int head, int c4,
+                                            const Merged& r) {
+    const float inv = r.l > 0.f ? 1.f / r.l : 0.f;
+    uint2 v;
+    v.x = pack_bf16(r.o.x * inv, r.o.y * inv);
+    v.y = pack_bf16(r.o.z * inv, r.o.w * inv);
+    *reinterpret_cast<uint2*>(p.out + (q_row * p.Hq + head) * kHeadDim + c4 * 4) = v;
+    if (p.lse && c4 == 0)
+        p.lse[q_row * p.Hq + head] = r.l > 0.f ? (r.m + log2f(r.l)) * 0.6931471805599453f : -INFINITY;
+}
+
+// Merge the splits of one group and write its final rows.  `tid` / `nthreads` enumerate the
+// calling threads; each handles (row, 4-column) cells.
+__device__ __forceinline__ void merge_group_splits(const AttnParams& p, const MergeGroup& g,
+                                                   int tid, int nthreads) {
+    const int rows = g.n_q * p.G;
+    const int64_t q_row0 = p.q_indptr ? p.q_indptr[g.seq] : g.seq;
+    for (int idx = tid; idx < rows * 32; idx += nthreads) {
+        const int R = idx >> 5, c4 = idx & 31;
+        const int64_t base = (int64_t)g.first_item * p.rows_cap + R;
+        const int64_t stride = p.rows_cap;
+        const float* ml = p.part_ml;
+        const float* po = p.part_o;
+        Merged r = merge_states(
+            g.n_splits,
+            [&](int i) { return __ldcg(ml + (base + i * stride) * 2); },
+            [&](int i) { return __ldcg(ml + (base + i * stride) * 2 + 1); },
+            [&](int i) {
+                return __ldcg(reinterpret_cast<const float4*>(po + (base + i * stride) * kHeadDim) + c4);
+            });
+        store_final(p, q_row0 + R / p.G, g.kv_head * p.G + R % p.G, c4, r);
+    }
+}
+
+// ------------------------------------------------------------------------------ the split kernel
+__global__ void __launch_bounds__(kThreads, 2)
+kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    // the 128-byte swizzle pattern repeats every 1024 bytes: tiles must start on that boundary
+    unsigned char* tiles = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    SmemTail* tail = reinterpret_cast<SmemTail*>(tiles + kStages * kStageBytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&tail->full[s]), 1);
+            mbar_init(smem_u32(&tail->empty[s]), kConsumerWarps);
+        }
+        tail->is_last = 0;
+        tail->timed_out = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map) : "memory");
+    }
+    // Programmatic dependent launch: everything above overlaps the previous kernel's tail; nothing
+    // below (work list, Q, KV, partials) is touched before the previous kernel has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    const WorkItem item = p.items[blockIdx.x];
+    const int n_pages = item.page_end - item.page_begin;
+    const int n_iters = (n_pages + kStagePages - 1) / kStagePages;
+    const int L = p.ctx_len[item.seq];
+    const int64_t list0 = (int64_t)p.list_indptr[item.seq] + item.page_begin;
+    const int64_t list_end = p.list_indptr[item.seq + 1];
+    const uint64_t deadline = global_ns() + kWaitBudgetNs;
+
+    // page ids of the slice -> shared memory (they gate every TMA address)
+    for (int i = tid; i < n_pages; i += kThreads) {
+        int32_t ph = 0;
+        bool ok = (list0 + i) < list_end;
+        if (ok) {
+            ph = p.phys_pages[list0 + i];
+            ok = ph >= 0 && ph < p.num_pool_pages;
+        }
+        if (!ok) { ph = 0; atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX); }
+        tail->phys[i] = ph;
+        tail->logical[i] = p.logical_pages && ok ? p.logical_pages[list0 + i] : item.page_begin + i;
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------------ producer warp
+        if (lane == 0) {
+            uint64_t policy;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+            const int rows_per_page = 2 * p.Hkv * kPageSize;
+            const int v_row_off = p.Hkv * kPageSize;
+            for (int it = 0; it < n_iters; ++it) {
+                const int s = it % kStages;
+                if (it >= kStages)
+                    mbar_wait(smem_u32(&tail->empty[s]), ((it / kStages) - 1) & 1, deadline,
+                              &tail->timed_out);
+                const int np = min(kStagePages, n_pages - it * kStagePages);
+                const uint32_t bar = smem_u32(&tail->full[s]);
+                mbar_expect_tx(bar, np * kPageHeadBytes);
+                for (int ps = 0; ps < np; ++ps) {
+                    const int y = tail->phys[it * kStagePages + ps] * rows_per_page
+                                  + item.kv_head * kPageSize;
+                    const uint32_t dst = smem_u32(tiles + s * kStageBytes + ps * kPageHeadBytes);
+                    tma_load_2d(dst, &kv_map, 0, y, bar, policy);
+                    tma_load_2d(dst + kHalfTileBytes, &kv_map, 64, y, bar, policy);
+                    tma_load_2d(dst + kTileBytes, &kv_map, 0, y + v_row_off, bar, policy);
+                    tma_load_2d(dst + kTileBytes + kHalfTileBytes, &kv_map, 64, y + v_row_off, bar,
+                                policy);
+                }
+            }
+        }
+        return;      // every load it issued is awaited by the consumers before they finish
+    }
+
+    // ---------------------------------------------------------------------- consumer warps
+    const int gid = lane >> 2, tid4 = lane & 3;
+    const int rows = item.n_q * p.G;                         // valid query rows of this item
+    int RT = (rows + kRowTile - 1) / kRowTile;               // row tiles: 1, 2 or 4
+    if (RT == 3) RT = 4;
+    const int rt = warp % RT;                                // this warp's row tile
+    const int ps0 = warp / RT, ps_step = kConsumerWarps / RT;
+    const int64_t q_row0 = p.q_indptr ? p.q_indptr[item.seq] : item.seq;
+
+    // Q fragments (A operand, 16 rows x 128) straight from global memory, zero for padding rows.
+    // Row R of the item = query token R / G, head R % G of the group.
+    uint32_t qf[8][4];
+    int pos_row[2];                                          // logical position of rows gid, gid+8
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        const int R = rt * kRowTile + gid + half * 8;
+        const bool valid = R < rows;
+        const int j = valid ? R / p.G : item.n_q - 1;
+        pos_row[half] = L - item.n_q + j;
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(
+            p.q + ((q_row0 + j) * p.Hq + item.kv_head * p.G + (valid ? R % p.G : 0)) * kHeadDim);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            qf[ks][half] = valid ? __ldg(src + ks * 8 + tid4) : 0u;          // cols 16ks + 2tid4
+            qf[ks][half + 2] = valid ? __ldg(src + ks * 8 + 4 + tid4) : 0u;  // cols 16ks + 8 + 2tid4
+        }
+    }
+
+    float o[16][4];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY};                 // running max (log2 units)
+    float l_run[2] = {0.f, 0.f};                             // this lane's share of the row sums
+    const float sc = p.scale_log2;
+    const int full_vis_limit = L - item.n_q;                 // tokens <= this are visible to all rows
+
+    // per-lane ldmatrix row addressing inside a tile (row = token, 128-byte rows, 16-byte chunk
+    // index xor (row & 7) = the TMA 128-byte swizzle)
+    const int lm = lane >> 3, lr = lane & 7;
+    const int k_tok = ((lm >> 1) << 3) + lr, k_cbit = lm & 1;   // K: matrices (n-tile, k-half)
+    const int v_tok = ((lm & 1) << 3) + lr, v_cbit = lm >> 1;   // V^T: matrices (k-half, n-tile)
+
+    for (int it = 0; it < n_iters; ++it) {
+        const int s = it % kStages;
+        mbar_wait(smem_u32(&tail->full[s]), (it / kStages) & 1, deadline, &tail->timed_out);
+        const int np = min(kStagePages, n_pages - it * kStagePages);
+        for (int ps = ps0; ps < np; ps += ps_step) {
+            const uint32_t kb = smem_u32(tiles + s * kStageBytes + ps * kPageHeadBytes);
+            const uint32_t vb = kb + kTileBytes;
+            const int tok0 = tail->logical[it * kStagePages + ps] * kPageSize;
+
+            // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
+            float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(kb + (ks >> 2) * kHalfTileBytes + k_tok * 128
+                           + ((((ks & 3) * 2 + k_cbit) ^ lr) << 4), b0, b1, b2, b3);
+                mma_bf16(sacc[0], qf[ks], b0, b1);
+                mma_bf16(sacc[1], qf[ks], b2, b3);
+            }
+            if (tok0 + kPageSize - 1 > full_vis_limit) {
+                // page reaches into the causal / tail region: mask per element
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int t = tok0 + nt * 8 + tid4 * 2 + (e & 1);
+                        if (t > pos_row[e >> 1]) sacc[nt][e] = -INFINITY;
+                    }
+                // value rows past the end of the context may hold anything (even NaN): zero them
+                const int first_bad = L - tok0;
+                if (first_bad < kPageSize) {
+                    if (lane < 16) {
+                        for (int r = max(first_bad, 0); r < kPageSize; ++r)
+                            *reinterpret_cast<uint4*>(tiles + s * kStageBytes + ps * kPageHeadBytes
+                                                      + kTileBytes + (lane >> 3) * kHalfTileBytes
+                                                      + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                }
+            }
+            // online softmax (base 2): rows gid (e = 0,1) and gid + 8 (e = 2,3)
+            float mx[2];
+            mx[0] = fmaxf(fmaxf(sacc[0][0], sacc[0][1]), fmaxf(sacc[1][0], sacc[1][1]));
+            mx[1] = fmaxf(fmaxf(sacc[0][2], sacc[0][3]), fmaxf(sacc[1][2], sacc[1][3]));
+            float corr[2], mu[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+                const float mn = fmaxf(m_run[h], mx[h] * sc);
+                mu[h] = (mn == -INFINITY) ? 0.f : mn;
+                corr[h] = ex2(m_run[h] - mu[h]);
+                m_run[h] = mn;
+            }
+            uint32_t pa[4];      // P as the A operand of P V (rows gid / gid+8, tokens 0-7 / 8-15)
+            pa[0] = pack_bf16(ex2(fmaf(sacc[0][0], sc, -mu[0])), ex2(fmaf(sacc[0][1], sc, -mu[0])));
+            pa[1] = pack_bf16(ex2(fmaf(sacc[0][2], sc, -mu[1])), ex2(fmaf(sacc[0][3], sc, -mu[1])));
+            pa[2] = pack_bf16(ex2(fmaf(sacc[1][0], sc, -mu[0])), ex2(fmaf(sacc[1][1], sc, -mu[0])));
+            pa[3] = pack_bf16(ex2(fmaf(sacc[1][2], sc, -mu[1])), ex2(fmaf(sacc[1][3], sc, -mu[1])));
+            // the row sums use the rounded weights, so out = sum(p v) / sum(p) is a true average
+            l_run[0] = fmaf(l_run[0], corr[0],
+                            (bf16_lo(pa[0]) + bf16_hi(pa[0])) + (bf16_lo(pa[2]) + bf16_hi(pa[2])));
+            l_run[1] = fmaf(l_run[1], corr[1],
+                            (bf16_lo(pa[1]) + bf16_hi(pa[1])) + (bf16_lo(pa[3]) + bf16_hi(pa[3])));
+            if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    o[i][0] *= corr[0]; o[i][1] *= corr[0];
+                    o[i][2] *= corr[1]; o[i][3] *= corr[1];
+                }
+            }
+            // O += P V   (16 n-tiles of 8 output columns, two per ldmatrix)
+#pragma unroll
+            for (int n2 = 0; n2 < 8; ++n2) {
+                uint32_t v0, v1, v2, v3;
+                ldsm_x4_t(vb + (n2 >> 2) * kHalfTileBytes + v_tok * 128
+                             + ((((n2 & 3) * 2 + v_cbit) ^ lr) << 4), v0, v1, v2, v3);
+                mma_bf16(o[2 * n2], pa, v0, v1);
+                mma_bf16(o[2 * n2 + 1], pa, v2, v3);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tail->empty[s]));
+    }
+    if (lane == 0 && tail->timed_out) atomicOr(p.status, 1 << KAP_ERR_TIMEOUT);
+
+    // ------------------------------------------------ combine the four warps' states, write out
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 1);
+        l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 2);
+    }
+    consumer_sync();                                   // all tile reads done: the ring is scratch now
+    float* scratch = reinterpret_cast<float*>(tiles) + warp * (kRowTile * kScratchStride);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        *reinterpret_cast<float2*>(scratch + gid * kScratchStride + i * 8 + tid4 * 2) =
+            make_float2(o[i][0], o[i][1]);
+        *reinterpret_cast<float2*>(scratch + (gid + 8) * kScratchStride + i * 8 + tid4 * 2) =
+            make_float2(o[i][2], o[i][3]);
+    }
+    if (tid4 == 0) {
+        tail->m[warp][gid] = m_run[0];     tail->l[warp][gid] = l_run[0];
+        tail->m[warp][gid + 8] = m_run[1]; tail->l[warp][gid + 8] = l_run[1];
+    }
+    consumer_sync();
+
+    const float* all = reinterpret_cast<const float*>(tiles);
+    const int n_same = kConsumerWarps / RT;            // warps that share a row tile
+    const bool single = item.n_splits == 1;
+    for (int idx = tid; idx < rows * 32; idx += kConsumerWarps * 32) {
+        const int R = idx >> 5, c4 = idx & 31;
+        const int t = R / kRowTile, r = R % kRowTile;
+        Merged res = merge_states(
+            n_same,
+            [&](int i) { return tail->m[t + i * RT][r]; },
+            [&](int i) { return tail->l[t + i * RT][r]; },
+            [&](int i) {
+                return *reinterpret_cast<const float4*>(
+                    all + ((t + i * RT) * kRowTile + r) * kScratchStride + c4 * 4);
+            });
+        if (single) {
+            store_final(p, q_row0 + R / p.G, item.kv_head * p.G + R % p.G, c4, res);
+        } else {
+            const int64_t prow = (int64_t)item.split * p.rows_cap + R;
+            *(reinterpret_cast<float4*>(p.part_o + prow * kHeadDim) + c4) = res.o;
+            if (c4 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(res.m, res.l);
+        }
+    }
+    if (single || !p.fused_merge) return;
+
+    // Fused merge: the last split of the group to arrive combines all of them.
+    __threadfence();
+    consumer_sync();
+    if (tid == 0) {
+        const int prev = atomicAdd(p.counters + item.group, 1);
+        const int last = prev == item.n_splits - 1;
+        if (last) p.counters[item.group] = 0;           // leave the counter clean for the next launch
+        tail->is_last = last;
+    }
+    consumer_sync();
+    if (!tail->is_last) return;
+    __threadfence();
+    merge_group_splits(p, p.groups[item.group], tid, kConsumerWarps * 32);
+}
+
+// -------------------------------------------------------------------- the separate merge kernel
+// One CTA per (sequence, KV head) that has more than one split.
+__global__ void __launch_bounds__(128)
+kap_attn_merge_kernel(const AttnParams p, const MergeGroup* merge_groups)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    merge_group_splits(p, merge_groups[blockIdx.x], threadIdx.x, blockDim.x);
+}
+
+// ================================================================================= host side
+namespace {
+
+std::atomic<long long> g_launches{0};
+std::atomic<int> g_use_pdl{1};
+std::atomic<int> g_fused_merge{0};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+#define KAP_CUDA(call)                                                                         \
+    do {                                                                                       \
+        cudaError_t e_ = (call);                                                               \
+        if (e_ != cudaSuccess)                                                                 \
+            return fail(KAP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));         \
+    } while (0)
+
+// Tensor map over one layer's pool viewed as a 2-D bf16 matrix [pages*2*Hkv*P rows][128 cols];
+// box = 16 rows x 64 columns (one half of a page-head's K or V), 128-byte swizzle.
+kap_status get_tensor_map(kap_workspace* ws, const void* pool, int64_t pages, int32_t hkv,
+                          const CUtensorMap** out) {
+    for (int i = 0; i < ws->map_count; ++i) {
+        auto& s = ws->maps[i];
+        if (s.base == pool && s.pages == pages && s.hkv == hkv) {
+            *out = reinterpret_cast<const CUtensorMap*>(s.map);
+            return KAP_OK;
+        }
+    }
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return fail(KAP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    const uint64_t rows = (uint64_t)pages * 2 * hkv * kPageSize;
+    if (rows >= (1ull << 31)) return fail(KAP_ERR_UNSUPPORTED, "pool of %lld pages is too large", (long long)pages);
+    cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kPageSize};
+    cuuint32_t estr[2] = {1, 1};
+    auto& slot = ws->maps[ws->map_next];
+    CUresult r = enc(reinterpret_cast<CUtensorMap*>(slot.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                     const_cast<void*>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(KAP_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
+    slot.base = pool; slot.pages = pages; slot.hkv = hkv;
+    *out = reinterpret_cast<const CUtensorMap*>(slot.map);
+    ws->map_next = (ws->map_next + 1) % kap_workspace::kMapSlots;
+    if (ws->map_count < kap_workspace::kMapSlots) ++ws->map_count;
+    return KAP_OK;
+}
+
+std::once_flag g_attr_once;
+cudaError_t g_attr_err = cudaSuccess;
+
+kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pages,
+                            kap_workspace* ws, cudaStream_t stream) {
+    if (ws->n_items == 0) return KAP_OK;
+    const CUtensorMap* map = nullptr;
+    kap_status st = get_tensor_map(ws, pool, pages, p_in.Hkv, &map);
+    if (st != KAP_OK) return st;
+    std::call_once(g_attr_once, [] {
+        g_attr_err = cudaFuncSetAttribute(kap_attn_split_kernel,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    });
+    if (g_attr_err != cudaSuccess)
+        return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(g_attr_err));
+
+    AttnParams p = p_in;
+    p.fused_merge = g_fused_merge.load() ? 1 : 0;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)ws->n_items);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_use_pdl.load() ? 1 : 0;
+    KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel, *map, p));
+    g_launches.fetch_add(1);
+    if (!p.fused_merge && ws->n_merge_groups > 0) {
+        cfg.gridDim = dim3((unsigned)ws->n_merge_groups);
+        cfg.blockDim = dim3(128);
+        cfg.dynamicSmemBytes = 0;
+        const MergeGroup* mg = ws->d_merge;
+        KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_merge_kernel, p, mg));
+        g_launches.fetch_add(1);
+    }
+    return KAP_OK;
+}
+
+kap_status check_shape(int32_t batch, int32_t hq, int32_t hkv, int32_t d, int32_t page,
+                       const kap_workspace* ws, const void* pool, bool verify) {
+    if (!ws) return fail(KAP_ERR_INVALID_ARG, "NULL workspace");
+    if (d != kHeadDim || page != kPageSize)
+        return fail(KAP_ERR_UNSUPPORTED, "head_dim %d / page_size %d (supported: 128 / 16)", d, page);
+    if (hq <= 0 || hkv <= 0 || hq % hkv || kRowTile % (hq / hkv))
+        return fail(KAP_ERR_UNSUPPORTED, "head counts %d / %d", hq, hkv);
+    if (batch != ws->batch || hq != ws->num_q_heads || hkv != ws->num_kv_heads)
+        return fail(KAP_ERR_INVALID_ARG, "call shape (batch %d, heads %d/%d) differs from the schedule "
+                    "(batch %d, heads %d/%d)", batch, hq, hkv, ws->batch, ws->num_q_heads, ws->num_kv_heads);
+    if (verify != (ws->has_nq != 0))
+        return fail(KAP_ERR_INVALID_ARG, verify ? "verification needs a schedule made with n_q"
+                                                : "the proposal path needs a schedule made without n_q");
+    if (reinterpret_cast<uintptr_t>(pool) & 15) return fail(KAP_ERR_INVALID_ARG, "kv_pool is not 16-byte aligned");
+    return KAP_OK;
+}
+
+}  // namespace
+}  // namespace kap
+
+using namespace kap;
+
+extern "C" kap_status kap_workspace_create(kap_workspace** out, int32_t device, int32_t max_items,
+                                           int32_t max_rows_per_item, int32_t max_batch) {
+    if (!out) return fail(KAP_ERR_INVALID_ARG, "NULL workspace pointer");
+    *out = nullptr;
+    if (max_items <= 0 || max_batch <= 0 || max_rows_per_item <= 0 ||
+        max_rows_per_item > kRowTile * kMaxRowTiles)
+        return fail(KAP_ERR_INVALID_ARG, "workspace sizes (%d items, %d rows, %d sequences)", max_items,
+                    max_rows_per_item, max_batch);
+    KAP_CUDA(cudaSetDevice(device));
+    cudaDeviceProp prop;
+    KAP_CUDA(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10)
+        return fail(KAP_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a only",
+                    device, prop.major, prop.minor);
+    auto* ws = new kap_workspace();
+    ws->device = device; ws->max_items = max_items; ws->max_rows = max_rows_per_item;
+    ws->max_batch = max_batch; ws->sm_count = prop.multiProcessorCount;
+    const size_t max_groups = (size_t)max_items;
+    cudaError_t e = cudaSuccess;
+    auto dev = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
+    auto host = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMallocHost(p, bytes); };
+    dev((void**)&ws->d_items, sizeof(WorkItem) * max_items);
+    dev((void**)&ws->d_groups, sizeof(MergeGroup) * max_groups);
+    dev((void**)&ws->d_merge, sizeof(MergeGroup) * max_groups);
+    dev((void**)&ws->d_part_o, sizeof(float) * (size_t)max_items * max_rows_per_item * kHeadDim);
+    dev((void**)&ws->d_part_ml, sizeof(float) * (size_t)max_items * max_rows_per_item * 2);
+    dev((void**)&ws->d_counters, sizeof(int32_t) * max_groups);
+    dev((void**)&ws->d_status, sizeof(int32_t));
+    host((void**)&ws->h_items, sizeof(WorkItem) * max_items);
+    host((void**)&ws->h_groups, sizeof(MergeGroup) * max_groups);
+    host((void**)&ws->h_merge, sizeof(MergeGroup) * max_groups);
+    host((void**)&ws->h_status, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ws->d_counters, 0, sizeof(int32_t) * max_groups);
+    if (e == cudaSuccess) e = cudaMemset(ws->d_status, 0, sizeof(int32_t));
+    cudaEvent_t ev = nullptr;
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+    ws->upload_event = ev;
+    ws->maps = new kap_workspace::MapSlot[kap_workspace::kMapSlots]();
+    if (e != cudaSuccess) {
+        kap_workspace_destroy(ws);
+        return fail(KAP_ERR_CUDA, "workspace allocation failed: %s", cudaGetErrorString(e));
+    }
+    // resident CTAs per SM decide how many items make one wave
+    int per_sm = 0;
+    cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kap_attn_split_kernel, kThreads,
+                                                      kSmemBytes) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    ws->ctas_per_wave = per_sm * ws->sm_count;
+    *out = ws;
+    return KAP_OK;
+}
+
+extern "C" void kap_workspace_destroy(kap_workspace* ws) {
+    if (!ws) return;
+    cudaFree(ws->d_items); cudaFree(ws->d_groups); cudaFree(ws->d_merge); cudaFree(ws->d_part_o);
+    cudaFree(ws->d_part_ml); cudaFree(ws->d_counters); cudaFree(ws->d_status);
+    cudaFreeHost(ws->h_items); cudaFreeHost(ws->h_groups); cudaFreeHost(ws->h_merge);
+    cudaFreeHost(ws->h_status);
+    if (ws->upload_event) cudaEventDestroy((cudaEvent_t)ws->upload_event);
+    delete[] ws->maps;
+    delete ws;
+}
+
+extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32_t* list_len,
+                                   const int32_t* n_q, int32_t num_q_heads, int32_t num_kv_heads,
+                                   int32_t max_chunk_pages, void* cuda_stream) {
+    if (!ws) return fail(KAP_ERR_INVALID_ARG, "NULL workspace");
+    if (batch > ws->max_batch) return fail(KAP_ERR_CAPACITY, "batch %d > workspace max_batch %d", batch, ws->max_batch);
+    std::vector<WorkItem> items;
+    std::vector<MergeGroup> groups;
+    int32_t max_chunk = 0, row_tiles = 1;
+    kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, ws->ctas_per_wave,
+                                   max_chunk_pages, ws->max_items, ws->max_rows, items, groups,
+                                   &max_chunk, &row_tiles);
+    if (st != KAP_OK) return st;
+    if ((int64_t)items.size() > ws->max_items || (int64_t)groups.size() > ws->max_items)
+        return fail(KAP_ERR_CAPACITY, "%zu work items exceed the workspace's %d", items.size(), ws->max_items);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // the pinned staging buffers may still feed the previous upload
+    KAP_CUDA(cudaEventSynchronize((cudaEvent_t)ws->upload_event));
+    int32_t n_merge = 0;
+    int64_t total_rows = 0;
+    for (int32_t b = 0; b < batch; ++b) total_rows += n_q ? n_q[b] : 1;
+    for (size_t i = 0; i < groups.size(); ++i) {
+        ws->h_groups[i] = groups[i];
+        if (groups[i].n_splits > 1) ws->h_merge[n_merge++] = groups[i];
+    }
+    if (!items.empty()) std::memcpy(ws->h_items, items.data(), sizeof(WorkItem) * items.size());
+    KAP_CUDA(cudaSetDevice(ws->device));
+    if (!items.empty()) {
+        KAP_CUDA(cudaMemcpyAsync(ws->d_items, ws->h_items, sizeof(WorkItem) * items.size(),
+                                 cudaMemcpyHostToDevice, stream));
+        KAP_CUDA(cudaMemcpyAsync(ws->d_groups, ws->h_groups, sizeof(MergeGroup) * groups.size(),
+                                 cudaMemcpyHostToDevice, stream));
+        if (n_merge)
+            KAP_CUDA(cudaMemcpyAsync(ws->d_merge, ws->h_merge, sizeof(MergeGroup) * n_merge,
+                                     cudaMemcpyHostToDevice, stream));
+    }
+    KAP_CUDA(cudaEventRecord((cudaEvent_t)ws->upload_event, stream));
+    ws->batch = batch; ws->n_items = (int32_t)items.size(); ws->n_groups = (int32_t)groups.size();
+    ws->n_merge_groups = n_merge; ws->max_chunk = max_chunk; ws->row_tiles = row_tiles;
+    ws->num_q_heads = num_q_heads; ws->num_kv_heads = num_kv_heads; ws->has_nq = n_q != nullptr;
+    ws->total_rows = total_rows;
+    return KAP_OK;
+}
+
+extern "C" kap_status kap_schedule_info(const kap_workspace* ws, int32_t* n_items,
+                                        int32_t* n_merge_groups, int32_t* max_chunk_pages,
+                                        int32_t* ctas_per_wave) {
+    if (!ws) return fail(KAP_ERR_INVALID_ARG, "NULL workspace");
+    if (n_items) *n_items = ws->n_items;
+    if (n_merge_groups) *n_merge_groups = ws->n_merge_groups;
+    if (max_chunk_pages) *max_chunk_pages = ws->max_chunk;
+    if (ctas_per_wave) *ctas_per_wave = ws->ctas_per_wave;
+    return KAP_OK;
+}
+
+static AttnParams base_params(kap_workspace* ws, int32_t hq, int32_t hkv, float sm_scale,
+                              int64_t num_pool_pages) {
+    AttnParams p{};
+    p.items = ws->d_items; p.groups = ws->d_groups; p.part_o = ws->d_part_o;
+    p.part_ml = ws->d_part_ml; p.counters = ws->d_counters; p.status = ws->d_status;
+    p.num_pool_pages = num_pool_pages; p.Hq = hq; p.Hkv = hkv; p.G = hq / hkv;
+    p.rows_cap = ws->max_rows;
+    p.scale_log2 = sm_scale * 1.4426950408889634f;
+    return p;
+}
+
+extern "C" kap_status kap_selected_decode_attn(
+    const void* q, const void* kv_pool, int64_t num_pool_pages, const int32_t* plan_indptr,
+    const int32_t* plan_phys_pages, const int32_t* plan_logical_pages, const int32_t* ctx_len,
+    int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
+    float sm_scale, void* out, float* lse, kap_workspace* ws, void* cuda_stream)
+{
+    kap_status st = check_shape(batch, num_q_heads, num_kv_heads, head_dim, page_size, ws, kv_pool, false);
+    if (st != KAP_OK) return st;
+    if (batch == 0) return KAP_OK;
+    if (!q || !kv_pool || !plan_indptr || !plan_phys_pages || !ctx_len || !out || num_pool_pages <= 0)
+        return fail(KAP_ERR_INVALID_ARG, "NULL pointer or empty pool");
+    AttnParams p = base_params(ws, num_q_heads, num_kv_heads, sm_scale, num_pool_pages);
+    p.q = (const __nv_bfloat16*)q; p.q_indptr = nullptr; p.list_indptr = plan_indptr;
+    p.phys_pages = plan_phys_pages; p.logical_pages = plan_logical_pages; p.ctx_len = ctx_len;
+    p.out = (__nv_bfloat16*)out; p.lse = lse;
+    return launch_attention(p, kv_pool, num_pool_pages, ws, (cudaStream_t)cuda_stream);
+}
+
+extern "C" kap_status kap_verify_attn(
+    const void* q, const int32_t* q_indptr, const void* kv_pool, int64_t num_pool_pages,
+    const int32_t* bt_indptr, const int32_t* bt_pages, const int32_t* ctx_len, int32_t batch,
+    int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t page_size, float sm_scale,
+    void* out, float* lse, kap_workspace* ws, void* cuda_stream)
+{
+    kap_status st = check_shape(batch, num_q_heads, num_kv_heads, head_dim, page_size, ws, kv_pool, true);
+    if (st != KAP_OK) return st;
+    if (batch == 0) return KAP_OK;
+    if (!q || !q_indptr || !kv_pool || !bt_indptr || !bt_pages || !ctx_len || !out || num_pool_pages <= 0)
+        return fail(KAP_ERR_INVALID_ARG, "NULL pointer or empty pool");
+    AttnParams p = base_params(ws, num_q_heads, num_kv_heads, sm_scale, num_pool_pages);
+    p.q = (const __nv_bfloat16*)q; p.q_indptr = q_indptr; p.list_indptr = bt_indptr;
+    p.phys_pages = bt_pages; p.logical_pages = nullptr; p.ctx_len = ctx_len;
+    p.out = (__nv_bfloat16*)out; p.lse = lse;
+    return launch_attention(p, kv_pool, num_pool_pages, ws, (cudaStream_t)cuda_stream);
+}
+
+extern "C" kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream) {
+    if (!ws) return fail(KAP_ERR_INVALID_ARG, "NULL workspace");
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    KAP_CUDA(cudaMemcpyAsync(ws->h_status, ws->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    KAP_CUDA(cudaMemsetAsync(ws->d_status, 0, sizeof(int32_t), stream));
+    KAP_CUDA(cudaStreamSynchronize(stream));
+    const int32_t s = *ws->h_status;
+    if (s & (1 << KAP_ERR_TIMEOUT)) return fail(KAP_ERR_TIMEOUT, "a device-side wait ran out");
+    if (s & (1 << KAP_ERR_DEVICE_INDEX)) return fail(KAP_ERR_DEVICE_INDEX, "a kernel met an out-of-range page or list index");
+    return KAP_OK;
+}
+
+extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t fused_merge) {
+    if (use_pdl >= 0) g_use_pdl.store(use_pdl ? 1 : 0);
+    if (fused_merge >= 0) g_fused_merge.store(fused_merge ? 1 : 0);
+    return KAP_OK;
+}
+
+extern "C" int64_t kap_launch_count(void) { return g_launches.load(); }

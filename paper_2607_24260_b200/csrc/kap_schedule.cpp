@@ -1,0 +1,159 @@
+// Split-K work scheduling for the attention kernels (host code, no GPU).
+//
+// The paper (Section 3.2, "Runtime stability and fallback") asks for stable metadata shapes so
+// that decode steps replay as CUDA graphs; it does not describe how one sequence's pages are
+// spread over a GPU.  This file is that part: every (sequence, KV head) page list is cut into
+// near-equal contiguous chunks, one chunk per CTA, such that the chunks fill the GPU's resident
+// CTA slots in whole waves.  The result depends only on page counts and row counts, so it is
+// computed once per request shape and reused for every layer and step.
+#include <algorithm>
+#include <cstring>
+#include <numeric>
+#include <vector>
+
+#include "kap_internal.h"
+
+namespace kap {
+
+namespace {
+
+// chunks needed when every list is cut into pieces of at most t pages
+int64_t chunks_for(const int32_t* len, int32_t batch, int32_t hkv, int64_t t) {
+    int64_t n = 0;
+    for (int32_t b = 0; b < batch; ++b) n += ((int64_t)len[b] + t - 1) / t;
+    return n * hkv;
+}
+
+}  // namespace
+
+// Cost model used to pick the number of waves: a CTA pays a fixed start-up/epilogue cost worth
+// about kFixedPages pages of streaming, waves run back to back.
+constexpr int64_t kFixedPages = 6;
+constexpr int32_t kDefaultChunkCap = 512;     // also the size of the kernel's page-id buffer
+
+kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t* n_q,
+                          int32_t num_q_heads, int32_t num_kv_heads, int32_t cta_slots,
+                          int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
+                          std::vector<WorkItem>& items, std::vector<MergeGroup>& groups,
+                          int32_t* max_chunk_out, int32_t* row_tiles_out)
+{
+    if (batch < 0 || (batch > 0 && !list_len)) return fail(KAP_ERR_INVALID_ARG, "bad batch / list_len");
+    if (num_q_heads <= 0 || num_kv_heads <= 0 || num_q_heads % num_kv_heads)
+        return fail(KAP_ERR_INVALID_ARG, "head counts %d / %d", num_q_heads, num_kv_heads);
+    const int32_t G = num_q_heads / num_kv_heads;
+    if (kRowTile % G) return fail(KAP_ERR_UNSUPPORTED, "group size %d must divide %d", G, kRowTile);
+    if (cta_slots <= 0) return fail(KAP_ERR_INVALID_ARG, "cta_slots %d", cta_slots);
+    int32_t cap = max_chunk_pages <= 0 ? kDefaultChunkCap : std::min(max_chunk_pages, kDefaultChunkCap);
+    int32_t max_len = 0, max_nq = 1;
+    for (int32_t b = 0; b < batch; ++b) {
+        if (list_len[b] <= 0) return fail(KAP_ERR_INVALID_ARG, "list_len[%d] = %d <= 0", b, list_len[b]);
+        const int32_t nq = n_q ? n_q[b] : 1;
+        if (nq < 1) return fail(KAP_ERR_INVALID_ARG, "n_q[%d] = %d < 1", b, nq);
+        max_len = std::max(max_len, list_len[b]);
+        max_nq = std::max(max_nq, nq);
+    }
+    const int32_t rows = max_nq * G;
+    if (rows > kRowTile * kMaxRowTiles)
+        return fail(KAP_ERR_UNSUPPORTED, "%d query rows per KV head exceed %d", rows, kRowTile * kMaxRowTiles);
+    if (rows > max_rows) return fail(KAP_ERR_CAPACITY, "%d rows per item, workspace holds %d", rows, max_rows);
+    int32_t row_tiles = (rows + kRowTile - 1) / kRowTile;
+    if (row_tiles == 3) row_tiles = 4;
+    items.clear();
+    groups.clear();
+    *max_chunk_out = 0;
+    *row_tiles_out = row_tiles;
+    if (batch == 0) return KAP_OK;
+
+    // smallest chunk size t with chunks_for(t) <= slots * waves, for the cheapest wave count
+    auto min_chunk = [&](int64_t budget) -> int64_t {
+        int64_t lo = 1, hi = max_len;
+        if (chunks_for(list_len, batch, num_kv_heads, hi) > budget) return -1;
+        while (lo < hi) {
+            const int64_t mid = (lo + hi) / 2;
+            if (chunks_for(list_len, batch, num_kv_heads, mid) <= budget) hi = mid; else lo = mid + 1;
+        }
+        return lo;
+    };
+    int64_t best_t = -1, best_cost = INT64_MAX;
+    const int64_t item_cap = std::max<int64_t>(1, max_items);
+    for (int64_t waves = 1; waves <= 64; ++waves) {
+        const int64_t budget = std::min<int64_t>(item_cap, (int64_t)cta_slots * waves);
+        const int64_t t = min_chunk(budget);
+        if (t > 0 && t <= cap) {
+            const int64_t cost = waves * (t + kFixedPages);
+            if (cost < best_cost) { best_cost = cost; best_t = t; }
+            if (t == 1) break;
+        }
+        if (budget == item_cap) break;                 // no further items to hand out
+    }
+    if (best_t < 0) {                                   // very long lists: as many items as allowed
+        const int64_t t = min_chunk(item_cap);
+        if (t > 0 && t <= cap) best_t = t;
+    }
+    if (best_t < 0)
+        return fail(KAP_ERR_CAPACITY, "page lists need more than %d work items of <= %d pages",
+                    max_items, cap);
+
+    int32_t slot = 0;
+    for (int32_t b = 0; b < batch; ++b) {
+        const int32_t len = list_len[b];
+        const int32_t n_splits = (int32_t)(((int64_t)len + best_t - 1) / best_t);
+        const int32_t base = len / n_splits, rem = len % n_splits;
+        for (int32_t g = 0; g < num_kv_heads; ++g) {
+            MergeGroup mg{};
+            mg.seq = b; mg.kv_head = g; mg.first_item = slot; mg.n_splits = n_splits;
+            mg.n_q = n_q ? n_q[b] : 1;
+            const int32_t group_index = (int32_t)groups.size();
+            groups.push_back(mg);
+            int32_t begin = 0;
+            for (int32_t s = 0; s < n_splits; ++s) {
+                const int32_t n = base + (s < rem ? 1 : 0);
+                WorkItem it{};
+                it.seq = b; it.kv_head = g; it.page_begin = begin; it.page_end = begin + n;
+                it.group = group_index; it.split = slot; it.n_splits = n_splits; it.n_q = mg.n_q;
+                items.push_back(it);
+                *max_chunk_out = std::max(*max_chunk_out, n);
+                begin += n;
+                ++slot;
+            }
+        }
+    }
+    // longest chunks first: the hardware hands out CTAs in index order, so the tail of the last
+    // wave is made of the shortest chunks.  WorkItem::split holds the item's partial-result slot
+    // (group.first_item + split index), which is what keeps a group's partials contiguous.
+    std::stable_sort(items.begin(), items.end(), [](const WorkItem& a, const WorkItem& c) {
+        return (a.page_end - a.page_begin) > (c.page_end - c.page_begin);
+    });
+    return KAP_OK;
+}
+
+}  // namespace kap
+
+// Exposed for tests and tools: the same schedule kap_schedule uploads, written to HOST arrays.
+// items_out holds max_items rows of 8 int32 (seq, kv_head, page_begin, page_end, group, slot,
+// n_splits, n_q).  Not a paper operation (see the file header).
+extern "C" kap_status kap_schedule_host(
+    int32_t batch, const int32_t* list_len, const int32_t* n_q, int32_t num_q_heads,
+    int32_t num_kv_heads, int32_t cta_slots, int32_t max_chunk_pages, int32_t max_items,
+    int32_t* items_out, int32_t* n_items, int32_t* n_merge_groups, int32_t* max_chunk)
+{
+    std::vector<kap::WorkItem> items;
+    std::vector<kap::MergeGroup> groups;
+    int32_t mc = 0, rt = 1;
+    kap_status st = kap::build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, cta_slots,
+                                        max_chunk_pages, max_items, kap::kRowTile * kap::kMaxRowTiles,
+                                        items, groups, &mc, &rt);
+    if (st != KAP_OK) return st;
+    if ((int64_t)items.size() > max_items)
+        return kap::fail(KAP_ERR_CAPACITY, "%zu items > max_items %d", items.size(), max_items);
+    if (items_out && !items.empty())
+        std::memcpy(items_out, items.data(), sizeof(kap::WorkItem) * items.size());
+    if (n_items) *n_items = (int32_t)items.size();
+    if (n_merge_groups) {
+        int32_t n = 0;
+        for (const auto& g : groups) n += g.n_splits > 1;
+        *n_merge_groups = n;
+    }
+    if (max_chunk) *max_chunk = mc;
+    return KAP_OK;
+}

@@ -1,0 +1,219 @@
+"""Thin Python binding of the C ABI in include/kap.h - argument marshalling only.
+
+Host-side calls take numpy arrays; the attention calls take torch CUDA tensors (PyTorch is used
+for device memory and streams only) and pass raw device pointers and the current CUDA stream.
+The shared library must have been built (``python -m paper_2607_24260_b200.build`` or
+``__graft_entry__.build()``); there is no fallback path: a missing library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_DEVICE_INDEX = range(7)
+PLAN_FULL, PLAN_OVER_BUDGET, PLAN_S_HIGH = 1, 2, 4
+
+_i32p, _f32p, _u8p, _vp = C.POINTER(C.c_int32), C.POINTER(C.c_float), C.POINTER(C.c_uint8), C.c_void_p
+
+# every symbol include/kap.h declares, with its signature
+SIGNATURES = {
+    "kap_compile_plan": (C.c_int, [C.c_int32, C.c_int32, _i32p, _i32p, _i32p, _i32p, _f32p, _i32p,
+                                   _i32p, _i32p, _u8p, C.c_float, _i32p, _i32p, C.c_int64, _i32p,
+                                   _i32p, _i32p, _i32p, _i32p]),
+    "kap_workspace_create": (C.c_int, [C.POINTER(_vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
+    "kap_workspace_destroy": (None, [_vp]),
+    "kap_schedule": (C.c_int, [_vp, C.c_int32, _i32p, _i32p, C.c_int32, C.c_int32, C.c_int32, _vp]),
+    "kap_schedule_host": (C.c_int, [C.c_int32, _i32p, _i32p, C.c_int32, C.c_int32, C.c_int32,
+                                    C.c_int32, C.c_int32, _i32p, _i32p, _i32p, _i32p]),
+    "kap_schedule_info": (C.c_int, [_vp, _i32p, _i32p, _i32p, _i32p]),
+    "kap_selected_decode_attn": (C.c_int, [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, C.c_int32,
+                                           C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float,
+                                           _vp, _vp, _vp, _vp]),
+    "kap_verify_attn": (C.c_int, [_vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_int32, C.c_int32,
+                                  C.c_int32, C.c_int32, C.c_int32, C.c_float, _vp, _vp, _vp, _vp]),
+    "kap_workspace_check": (C.c_int, [_vp, _vp]),
+    "kap_set_launch_options": (C.c_int, [C.c_int32, C.c_int32]),
+    "kap_launch_count": (C.c_int64, []),
+    "kap_last_error": (C.c_char_p, []),
+    "kap_version": (C.c_char_p, []),
+}
+
+_lib = None
+
+
+class KapError(RuntimeError):
+    def __init__(self, code, message):
+        super().__init__(f"kap status {code}: {message}")
+        self.code = code
+
+
+def lib():
+    """Load libkap_b200.so (built in-tree).  Raises if it is missing: there is no fallback."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path):
+            raise ImportError(f"{path} is missing: build it with `python -m paper_2607_24260_b200.build`")
+        handle = C.CDLL(path)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _check(code):
+    if code != OK:
+        raise KapError(code, lib().kap_last_error().decode())
+
+
+def _np(a, dt):
+    return None if a is None else np.ascontiguousarray(a, dtype=dt)
+
+
+def _ptr(a, ct):
+    return None if a is None else a.ctypes.data_as(C.POINTER(ct))
+
+
+def version() -> str:
+    return lib().kap_version().decode()
+
+
+def launch_count() -> int:
+    return int(lib().kap_launch_count())
+
+
+def set_launch_options(use_pdl: int = -1, fused_merge: int = -1):
+    _check(lib().kap_set_launch_options(int(use_pdl), int(fused_merge)))
+
+
+# ------------------------------------------------------------------------------- kap_compile_plan
+def compile_plan(ctx_len, span_indptr, span_start, span_len, span_score, budget_tokens, n_sink,
+                 n_recent, force_full=None, s_max=1.0, bt_indptr=None, bt_pages=None, page_size=16,
+                 capacity=None):
+    """kap_compile_plan on host arrays.  Returns a dict: plan_indptr, plan_logical_pages,
+    plan_phys_pages (None without a block table), plan_flags, selected_tokens."""
+    ctx_len = _np(ctx_len, np.int32)
+    B = int(ctx_len.shape[0])
+    span_indptr, span_start = _np(span_indptr, np.int32), _np(span_start, np.int32)
+    span_len, span_score = _np(span_len, np.int32), _np(span_score, np.float32)
+    budget_tokens, n_sink = _np(budget_tokens, np.int32), _np(n_sink, np.int32)
+    n_recent, force_full = _np(n_recent, np.int32), _np(force_full, np.uint8)
+    bt_indptr, bt_pages = _np(bt_indptr, np.int32), _np(bt_pages, np.int32)
+    if capacity is None:
+        capacity = int(sum((max(int(L), 0) + page_size - 1) // max(page_size, 1) for L in ctx_len))
+    indptr = np.full(B + 1, -1, dtype=np.int32)
+    logical = np.full(max(1, capacity), -1, dtype=np.int32)
+    phys = np.full(max(1, capacity), -1, dtype=np.int32) if bt_indptr is not None else None
+    flags = np.full(B, -1, dtype=np.int32)
+    sel = np.full(B, -1, dtype=np.int32)
+    _check(lib().kap_compile_plan(
+        B, page_size, _ptr(ctx_len, C.c_int32), _ptr(span_indptr, C.c_int32),
+        _ptr(span_start, C.c_int32), _ptr(span_len, C.c_int32), _ptr(span_score, C.c_float),
+        _ptr(budget_tokens, C.c_int32), _ptr(n_sink, C.c_int32), _ptr(n_recent, C.c_int32),
+        _ptr(force_full, C.c_uint8), float(s_max), _ptr(bt_indptr, C.c_int32),
+        _ptr(bt_pages, C.c_int32), int(capacity), _ptr(indptr, C.c_int32), _ptr(logical, C.c_int32),
+        _ptr(phys, C.c_int32), _ptr(flags, C.c_int32), _ptr(sel, C.c_int32)))
+    n = int(indptr[-1])
+    return dict(plan_indptr=indptr, plan_logical_pages=logical[:n].copy(),
+                plan_phys_pages=None if phys is None else phys[:n].copy(), plan_flags=flags,
+                selected_tokens=sel)
+
+
+def compile_workload(w, capacity=None):
+    """kap_compile_plan on a synth.Workload."""
+    return compile_plan(w.ctx_len, w.span_indptr, w.span_start, w.span_len, w.span_score,
+                        w.budget_tokens, w.n_sink, w.n_recent, w.force_full, w.s_max, w.bt_indptr,
+                        w.bt_pages, w.page_size, capacity)
+
+
+def schedule_host(list_len, n_q, num_q_heads, num_kv_heads, cta_slots, max_chunk_pages=0,
+                  max_items=8192):
+    """kap_schedule_host: the split-K work list as an [n_items, 8] int32 array (seq, kv_head,
+    page_begin, page_end, group, slot, n_splits, n_q) plus (n_merge_groups, max_chunk)."""
+    list_len = _np(list_len, np.int32)
+    n_q = _np(n_q, np.int32)
+    items = np.zeros((max_items, 8), dtype=np.int32)
+    n_items, n_merge, max_chunk = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    _check(lib().kap_schedule_host(int(list_len.shape[0]), _ptr(list_len, C.c_int32),
+                                   _ptr(n_q, C.c_int32), num_q_heads, num_kv_heads, cta_slots,
+                                   max_chunk_pages, max_items, _ptr(items, C.c_int32),
+                                   C.byref(n_items), C.byref(n_merge), C.byref(max_chunk)))
+    return items[:n_items.value].copy(), n_merge.value, max_chunk.value
+
+
+# ------------------------------------------------------------------------- workspace + attention
+def _stream_ptr(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _dptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+class Workspace:
+    """kap_workspace: split-K schedule + partial-result buffers for one launch shape."""
+
+    def __init__(self, device=0, max_items=8192, max_rows_per_item=16, max_batch=256):
+        self._h = C.c_void_p()
+        self.device = int(device)
+        _check(lib().kap_workspace_create(C.byref(self._h), self.device, max_items,
+                                          max_rows_per_item, max_batch))
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().kap_workspace_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def schedule(self, list_len, n_q=None, num_q_heads=32, num_kv_heads=8, max_chunk_pages=0,
+                 stream=None):
+        list_len = _np(list_len, np.int32)
+        n_q = _np(n_q, np.int32)
+        _check(lib().kap_schedule(self._h, int(list_len.shape[0]), _ptr(list_len, C.c_int32),
+                                  _ptr(n_q, C.c_int32), num_q_heads, num_kv_heads, max_chunk_pages,
+                                  _stream_ptr(stream)))
+        return self.info()
+
+    def info(self):
+        v = [C.c_int32(0) for _ in range(4)]
+        _check(lib().kap_schedule_info(self._h, *[C.byref(x) for x in v]))
+        return dict(n_items=v[0].value, n_merge_groups=v[1].value, max_chunk_pages=v[2].value,
+                    ctas_per_wave=v[3].value)
+
+    def check(self, stream=None):
+        _check(lib().kap_workspace_check(self._h, _stream_ptr(stream)))
+
+
+def selected_decode_attn(q, kv_pool, plan_indptr, plan_phys_pages, plan_logical_pages, ctx_len, out,
+                         ws: Workspace, lse=None, sm_scale=None, stream=None):
+    """kap_selected_decode_attn on torch CUDA tensors: q/out bf16 [B, Hq, d]; kv_pool bf16
+    [pages, 2, Hkv, P, d]; plan arrays and ctx_len int32 device tensors."""
+    B, Hq, d = q.shape
+    pages, _, Hkv, P, _ = kv_pool.shape
+    sm_scale = float(d) ** -0.5 if sm_scale is None else float(sm_scale)
+    _check(lib().kap_selected_decode_attn(
+        _dptr(q), _dptr(kv_pool), int(pages), _dptr(plan_indptr), _dptr(plan_phys_pages),
+        _dptr(plan_logical_pages), _dptr(ctx_len), B, Hq, Hkv, d, P, sm_scale, _dptr(out),
+        _dptr(lse), ws._h, _stream_ptr(stream)))
+    return out
+
+
+def verify_attn(q, q_indptr, kv_pool, bt_indptr, bt_pages, ctx_len, out, ws: Workspace, lse=None,
+                sm_scale=None, stream=None):
+    """kap_verify_attn on torch CUDA tensors: q/out bf16 [sum n_q, Hq, d]."""
+    _, Hq, d = q.shape
+    pages, _, Hkv, P, _ = kv_pool.shape
+    sm_scale = float(d) ** -0.5 if sm_scale is None else float(sm_scale)
+    _check(lib().kap_verify_attn(
+        _dptr(q), _dptr(q_indptr), _dptr(kv_pool), int(pages), _dptr(bt_indptr), _dptr(bt_pages),
+        _dptr(ctx_len), int(ctx_len.shape[0]), Hq, Hkv, d, P, sm_scale, _dptr(out), _dptr(lse),
+        ws._h, _stream_ptr(stream)))
+    return out
