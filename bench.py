@@ -1,0 +1,503 @@
+#!/usr/bin/env python
+"""Benchmark of the KAP hot path on B200: plan-guided decode attention tokens/s and HBM GB/s.
+
+A *step* is one propose-k / verify cycle of GraphSpec-style self-speculation (Section 3.2 and the
+cost model of Section 4.1, Eq. 7) over one batch, attention only: k selected-KV proposal passes
+(every layer: split-K kernel + merge) followed by one full-context verification pass with n_q = k
+rows (every layer).  Context length is held constant inside a cycle, as the paper's cost model
+assumes.  `value` = B*k proposed tokens per cycle / cycle time, inputs resident in HBM, the whole
+cycle replayed as two CUDA graphs (proposal segment, verification segment) with CUDA events
+between them.  `e2e` = the same cycle driven from HOST buffers through the C ABI: plan
+compilation and scheduling on the host, host->device copies of plan arrays and queries,
+device->host copy of every attention output, all inside the timed region (the KV cache itself is
+persistent state and stays on the device).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--no-sweep]
+    python bench.py --impl reference ...      # the CPU oracle on the same metric (rank 0 only)
+
+N > 1: one process per GPU (torchrun), every rank runs its own batch (weak scaling, no data-path
+collective); time = max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "plan-guided decode attn tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read+write per launch / algorithmic bytes per launch, from the ncu captures
+# summarised under profiles/ (kernel kap_attn_split_kernel); None until captured
+TRAFFIC_RATIO = {"decode": None, "verify": None}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------- clock sampler
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def __enter__(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.file is None:
+            return out
+        try:
+            self.file.flush()
+            with open(self.file.name) as f:
+                rows = [r.strip().split(", ") for r in f if r.strip()]
+            os.unlink(self.file.name)
+        except Exception:
+            return out
+        sm, reasons = [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                out["sm_max_mhz"] = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(names, r[4:8]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# -------------------------------------------------------------------------------- the GPU workload
+class Cycle:
+    """Device-resident state of one configuration plus the graphs that replay a cycle."""
+
+    def __init__(self, name, seed, layers=None, device="cuda:0", fused_merge=None):
+        import torch
+        from paper_2607_24260_b200 import kap, synth
+        self.torch, self.kap, self.synth = torch, kap, synth
+        self.dev = device
+        kw = {} if layers is None or name == "c1" else {"layers": layers}
+        self.w = w = synth.CONFIGS[name](seed, **kw)
+        self.k = int(w.n_q.max())                      # proposal steps per cycle
+        self.layers = w.layers
+        B, Hq, Hkv, d, P = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size
+        self.plan = kap.compile_workload(w)
+        self.n_sel = np.diff(self.plan["plan_indptr"])
+        self.n_pages = (w.ctx_len.astype(np.int64) + P - 1) // P
+        self.decode_bytes = int(self.n_sel.sum()) * w.page_bytes          # per layer, per pass
+        self.verify_bytes = int(self.n_pages.sum()) * w.page_bytes
+        # KV pool: one slice per layer so that no layer's KV is L2-resident when it is read
+        self.pool = torch.empty((self.layers, w.num_pool_pages, 2, Hkv, P, d),
+                                dtype=torch.bfloat16, device=device)
+        synth.device_fill_normal_(self.pool, 0.5, seed + 1)
+        rows_v = int(w.n_q.sum())
+        self.q_dec = torch.randn((self.k, self.layers, B, Hq, d), device=device,
+                                 generator=self._gen(seed + 2)).to(torch.bfloat16)
+        self.q_ver = torch.randn((self.layers, rows_v, Hq, d), device=device,
+                                 generator=self._gen(seed + 3)).to(torch.bfloat16)
+        self.out_dec = torch.zeros_like(self.q_dec)
+        self.out_ver = torch.zeros_like(self.q_ver)
+        i32 = lambda a: torch.from_numpy(np.array(a, dtype=np.int32)).to(device)
+        self.d_plan_indptr = i32(self.plan["plan_indptr"])
+        self.d_plan_phys = i32(self.plan["plan_phys_pages"])
+        self.d_plan_logical = i32(self.plan["plan_logical_pages"])
+        self.d_ctx = i32(w.ctx_len)
+        self.d_q_indptr = i32(w.q_indptr)
+        self.d_bt_indptr = i32(w.bt_indptr)
+        self.d_bt_pages = i32(w.bt_pages)
+        max_rows = int(w.n_q.max()) * (Hq // Hkv)
+        self.ws_d = kap.Workspace(int(device.split(":")[1]), 8192, Hq // Hkv, B)
+        self.ws_v = kap.Workspace(int(device.split(":")[1]), 8192, max_rows, B)
+        self.info_d = self.ws_d.schedule(self.n_sel, None, Hq, Hkv)
+        self.info_v = self.ws_v.schedule(self.n_pages, w.n_q, Hq, Hkv)
+        self.graph_d = self.graph_v = None
+        self.launches_per_step = 0
+
+    def _gen(self, seed):
+        g = self.torch.Generator(device=self.dev)
+        g.manual_seed(seed)
+        return g
+
+    # the two segments of a cycle, as plain enqueues (capturable)
+    def enqueue_proposal(self):
+        kap = self.kap
+        for step in range(self.k):
+            for layer in range(self.layers):
+                kap.selected_decode_attn(self.q_dec[step, layer], self.pool[layer], self.d_plan_indptr,
+                                         self.d_plan_phys, self.d_plan_logical, self.d_ctx,
+                                         self.out_dec[step, layer], self.ws_d)
+
+    def enqueue_verify(self):
+        kap = self.kap
+        for layer in range(self.layers):
+            kap.verify_attn(self.q_ver[layer], self.d_q_indptr, self.pool[layer], self.d_bt_indptr,
+                            self.d_bt_pages, self.d_ctx, self.out_ver[layer], self.ws_v)
+
+    def capture(self):
+        torch, kap = self.torch, self.kap
+        stream = torch.cuda.Stream(device=self.dev)
+        stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(stream):          # warm-up: tensor maps, function attributes
+            self.enqueue_proposal()
+            self.enqueue_verify()
+        stream.synchronize()
+        before = kap.launch_count()
+        self.graph_d = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph_d, stream=stream):
+            self.enqueue_proposal()
+        self.graph_v = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph_v, stream=stream):
+            self.enqueue_verify()
+        self.launches_per_step = kap.launch_count() - before
+        torch.cuda.synchronize()
+        self.ws_d.check()
+        self.ws_v.check()
+
+    def time_steps(self, steps, warmup):
+        """Returns (total_ms, decode_segment_ms, verify_segment_ms) over `steps` cycles."""
+        torch = self.torch
+        for _ in range(warmup):
+            self.graph_d.replay()
+            self.graph_v.replay()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+        torch.cuda.synchronize()
+        for s in range(steps):
+            ev[s][0].record()
+            self.graph_d.replay()
+            ev[s][1].record()
+            self.graph_v.replay()
+            ev[s][2].record()
+        torch.cuda.synchronize()
+        total = ev[0][0].elapsed_time(ev[-1][2])
+        dec = sum(e[0].elapsed_time(e[1]) for e in ev)
+        ver = sum(e[1].elapsed_time(e[2]) for e in ev)
+        return total, dec, ver
+
+    def free(self):
+        for ws in (self.ws_d, self.ws_v):
+            ws.close()
+        self.graph_d = self.graph_v = None
+        self.pool = self.q_dec = self.q_ver = self.out_dec = self.out_ver = None
+        self.torch.cuda.empty_cache()
+
+
+def summarise(cy: Cycle, steps, total_ms, dec_ms, ver_ms, n_ranks=1):
+    w = cy.w
+    peak, peak_kind = measured_peak()
+    ms_step = total_ms / steps
+    us_dec_layer = dec_ms / steps / (cy.k * cy.layers) * 1e3
+    us_ver_layer = ver_ms / steps / cy.layers * 1e3
+    gbs_dec = cy.decode_bytes / (us_dec_layer * 1e-6) / 1e9
+    gbs_ver = cy.verify_bytes / (us_ver_layer * 1e-6) / 1e9
+
+    def roof(kind, gbs, alg_bytes):
+        ratio = TRAFFIC_RATIO[kind]
+        return {"bound": "hbm", "kernel": f"kap_attn_split_kernel ({kind} launch incl. its merge pass)",
+                "achieved": round(gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(gbs / peak, 4),
+                "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4), "peak_kind": f"of {peak_kind}",
+                "algorithmic_bytes_per_launch": alg_bytes,
+                "traffic": None if ratio is None else int(ratio * alg_bytes)}
+
+    return {
+        "ms_per_step": ms_step,
+        "tokens_per_s": n_ranks * w.batch * cy.k / (ms_step * 1e-3),
+        "decode_only_tokens_per_s": n_ranks * w.batch / (dec_ms / steps / cy.k * 1e-3),
+        "us_per_layer_decode": round(us_dec_layer, 3),
+        "us_per_layer_verify": round(us_ver_layer, 3),
+        "decode": roof("decode", gbs_dec, cy.decode_bytes),
+        "verify": roof("verify", gbs_ver, cy.verify_bytes),
+        "share_decode": dec_ms / (dec_ms + ver_ms),
+        "retained_kv_ratio_s": float(cy.n_sel.sum() / cy.n_pages.sum()),
+        "schedule": {"decode": cy.info_d, "verify": cy.info_v},
+    }
+
+
+# ------------------------------------------------------------------------------------------- e2e
+def time_e2e(cy: Cycle, steps, warmup):
+    """The same cycle through the C ABI from HOST buffers: compile + schedule on the host, pinned
+    host -> device copies of the plan arrays, context lengths and every query, the two graph
+    segments, device -> host copies of every attention output; synchronised per step."""
+    torch, kap, w = cy.torch, cy.kap, cy.w
+    pin = lambda t: torch.empty(t.shape, dtype=t.dtype).pin_memory()
+    h_q_dec, h_q_ver = pin(cy.q_dec), pin(cy.q_ver)
+    h_q_dec.copy_(cy.q_dec)
+    h_q_ver.copy_(cy.q_ver)
+    h_out_dec, h_out_ver = pin(cy.out_dec), pin(cy.out_ver)
+    cap = int(cy.n_pages.sum())
+    h_indptr = torch.zeros(w.batch + 1, dtype=torch.int32).pin_memory()
+    h_phys = torch.zeros(cap, dtype=torch.int32).pin_memory()
+    h_logical = torch.zeros(cap, dtype=torch.int32).pin_memory()
+    h_ctx = torch.from_numpy(w.ctx_len.copy()).pin_memory()
+    n_plan = int(cy.plan["plan_indptr"][-1])
+    h2d = (h_q_dec.numel() + h_q_ver.numel()) * 2 + (h_indptr.numel() + 2 * n_plan + h_ctx.numel()) * 4
+    d2h = (h_out_dec.numel() + h_out_ver.numel()) * 2
+
+    def one_step():
+        plan = kap.compile_workload(w)                      # host: Algorithm 1
+        n = int(plan["plan_indptr"][-1])
+        h_indptr.numpy()[:] = plan["plan_indptr"]
+        h_phys.numpy()[:n] = plan["plan_phys_pages"]
+        h_logical.numpy()[:n] = plan["plan_logical_pages"]
+        cy.ws_d.schedule(np.diff(plan["plan_indptr"]), None, w.num_q_heads, w.num_kv_heads)
+        cy.ws_v.schedule(cy.n_pages, w.n_q, w.num_q_heads, w.num_kv_heads)
+        cy.d_plan_indptr.copy_(h_indptr, non_blocking=True)
+        cy.d_plan_phys[:n].copy_(h_phys[:n], non_blocking=True)
+        cy.d_plan_logical[:n].copy_(h_logical[:n], non_blocking=True)
+        cy.d_ctx.copy_(h_ctx, non_blocking=True)
+        cy.q_dec.copy_(h_q_dec, non_blocking=True)
+        cy.q_ver.copy_(h_q_ver, non_blocking=True)
+        cy.graph_d.replay()
+        cy.graph_v.replay()
+        h_out_dec.copy_(cy.out_dec, non_blocking=True)
+        h_out_ver.copy_(cy.out_ver, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        one_step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one_step()
+    torch.cuda.synchronize()
+    return (time.perf_counter() - t0) * 1e3 / steps, h2d, d2h
+
+
+# ---------------------------------------------------------------------------------- CPU baseline
+def oracle_cycle_seconds(w, plan, layers_budget_s=12.0, seed=0):
+    """Time the oracle, as it stands, on a bounded sample: whole layers of the workload (proposal
+    pass over all sequences + verification pass over all sequences), until about
+    `layers_budget_s` seconds of CPU work; returns (seconds per layer proposal, seconds per layer
+    verification, layers sampled, threads)."""
+    from oracle import kap_oracle as orc
+    from paper_2607_24260_b200 import synth
+    t_dec = t_ver = 0.0
+    n = 0
+    started = time.perf_counter()
+    while True:
+        q_bits, pool_bits = synth.host_qkv(w, seed, layer=n)
+        qd = q_bits[w.q_indptr[1:] - 1]
+        t0 = time.perf_counter()
+        orc.selected_decode_attn(qd, pool_bits, plan["plan_indptr"], plan["plan_phys_pages"],
+                                 plan["plan_logical_pages"], w.ctx_len)
+        t1 = time.perf_counter()
+        orc.verify_attn(q_bits, w.q_indptr, pool_bits, w.bt_indptr, w.bt_pages, w.ctx_len)
+        t2 = time.perf_counter()
+        t_dec += t1 - t0
+        t_ver += t2 - t1
+        n += 1
+        if (t_dec + t_ver) >= layers_budget_s or n >= w.layers or time.perf_counter() - started > 90:
+            break
+    return t_dec / n, t_ver / n, n, orc.num_threads()
+
+
+def cpu_baseline(w, k, budget_s=12.0):
+    from oracle import kap_oracle as orc
+    plan = orc.compile_workload(w)          # the oracle's own plan: nothing here comes from the library
+    t_dec, t_ver, n, threads = oracle_cycle_seconds(w, plan, budget_s)
+    cycle_s = w.layers * (k * t_dec + t_ver)
+    return {"value": w.batch * k / cycle_s, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+            "sample": f"{n} of {w.layers} layers of {w.name} (proposal pass + verification pass over all "
+                      f"{w.batch} sequences, fp64 C oracle, OpenMP), scaled to a {k}-proposal cycle over "
+                      f"{w.layers} layers",
+            "s_per_layer_decode": t_dec, "s_per_layer_verify": t_ver}
+
+
+# ------------------------------------------------------------------------------------------ main
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), \
+        int(os.environ.get("WORLD_SIZE", 1))
+
+
+def config_dict(w, k, layers, extra=None):
+    c = {"workload": f"{w.name}: {w.note}", "batch": w.batch, "ctx_len_max": int(w.ctx_len.max()),
+         "ctx_len_min": int(w.ctx_len.min()), "layers": layers, "proposals_per_cycle_k": k,
+         "verify_rows": k, "heads": f"{w.num_q_heads}q/{w.num_kv_heads}kv", "head_dim": w.head_dim,
+         "page_size": w.page_size,
+         "l2": "no flush: every layer has its own KV slice, per-cycle working set >> 126 MB L2"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the same metric and workload (rank 0 only)."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    from paper_2607_24260_b200 import synth
+    from oracle import kap_oracle as orc
+    w = synth.CONFIGS[args.config](0)
+    plan = orc.compile_workload(w)
+    k = int(w.n_q.max())
+    per_step_budget = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, sample = [], None
+    for i in range(args.warmup + args.steps):
+        t_dec, t_ver, n, threads = oracle_cycle_seconds(w, plan, per_step_budget, seed=i)
+        cycle_s = w.layers * (k * t_dec + t_ver)
+        if i >= args.warmup:
+            vals.append(cycle_s)
+        sample = f"{n} of {w.layers} layers per step, scaled to the full cycle"
+    ms = statistics.mean(vals) * 1e3
+    value = w.batch * k / (ms * 1e-3)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": config_dict(w, k, w.layers),
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--layers", type=int, default=None, help="override the layer count (debugging)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the 32K / 128K side measurements")
+    ap.add_argument("--sweep-layers", type=int, default=8)
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--fused-merge", type=int, default=-1)
+    ap.add_argument("--pdl", type=int, default=-1)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2607_24260_b200 import kap
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        from paper_2607_24260_b200 import dist as kdist
+        dist = kdist.Group("nccl", device=dev)
+    kap.set_launch_options(args.pdl, args.fused_merge)
+    warmup = max(3, args.warmup)
+
+    cy = Cycle(args.config, seed=rank, layers=args.layers, device=dev)
+    cy.capture()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local_rank) as clocks:
+        total_ms, dec_ms, ver_ms = cy.time_steps(args.steps, warmup)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+        total_ms = dist.max_float(total_ms)
+    res = summarise(cy, args.steps, total_ms, dec_ms, ver_ms, n_ranks=world)
+    e2e_ms, h2d, d2h = time_e2e(cy, max(3, min(args.steps, 20)), 3)
+    if dist:
+        e2e_ms = dist.max_float(e2e_ms)
+    cy.ws_d.check()
+    cy.ws_v.check()
+    w, k = cy.w, cy.k
+    dominant = "verify" if res["share_decode"] < 0.5 else "decode"
+    line = {
+        "metric": METRIC, "value": res["tokens_per_s"], "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": res["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": config_dict(w, k, cy.layers, {"parallelism": f"dp{world} (independent batches per GPU)",
+                                                 "pdl": args.pdl, "fused_merge": args.fused_merge}),
+        "clocks": clocks.summary(),
+        "e2e": {"value": world * w.batch * k / (e2e_ms * 1e-3), "unit": "tokens/s",
+                "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "note": "host plan compile + schedule + H2D of plans/queries + cycle + D2H of outputs; "
+                        "the KV cache is device-resident state"},
+        "gpu_launches": cy.launches_per_step * args.steps,
+        "roofline": res[dominant], "roofline_decode": res["decode"], "roofline_verify": res["verify"],
+        "us_per_layer_decode": res["us_per_layer_decode"],
+        "us_per_layer_verify": res["us_per_layer_verify"],
+        "decode_only_tokens_per_s": res["decode_only_tokens_per_s"],
+        "retained_kv_ratio_s": res["retained_kv_ratio_s"], "schedule": res["schedule"],
+    }
+    cy.free()
+
+    if rank == 0 and world == 1 and not args.no_sweep and args.config == "c2":
+        sweep = {}
+        for name in ("c3", "c4"):
+            try:
+                c2 = Cycle(name, seed=0, layers=args.sweep_layers, device=dev)
+                c2.capture()
+                t, d, v = c2.time_steps(max(5, args.steps // 4), 3)
+                r = summarise(c2, max(5, args.steps // 4), t, d, v)
+                sweep[name] = {"workload": c2.w.note, "layers_timed": c2.layers,
+                               "us_per_layer_decode": r["us_per_layer_decode"],
+                               "us_per_layer_verify": r["us_per_layer_verify"],
+                               "decode_GBps": r["decode"]["achieved"], "verify_GBps": r["verify"]["achieved"],
+                               "decode_frac_of_measured": r["decode"]["frac"],
+                               "decode_frac_of_8TBs": r["decode"]["frac_of_nominal_8TBs"],
+                               "verify_frac_of_measured": r["verify"]["frac"],
+                               "verify_frac_of_8TBs": r["verify"]["frac_of_nominal_8TBs"],
+                               "retained_kv_ratio_s": r["retained_kv_ratio_s"],
+                               "decode_only_tokens_per_s": r["decode_only_tokens_per_s"]}
+                c2.free()
+            except Exception as e:       # a side measurement must not lose the main line
+                sweep[name] = {"error": repr(e)}
+        line["sweep"] = sweep
+    if rank == 0 and world == 1 and not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(w, k)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist:
+        dist.close()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
