@@ -410,6 +410,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--fused-merge", type=int, default=-1)
     ap.add_argument("--pdl", type=int, default=-1)
+    ap.add_argument("--ctas-per-sm", type=int, default=-1)
+    ap.add_argument("--early-kv", type=int, default=-1)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -425,7 +427,7 @@ def main():
     if world > 1:
         from paper_2607_24260_b200 import dist as kdist
         dist = kdist.Group("nccl", device=dev)
-    kap.set_launch_options(args.pdl, args.fused_merge)
+    kap.set_launch_options(args.pdl, args.fused_merge, args.ctas_per_sm, args.early_kv)
     warmup = max(3, args.warmup)
 
     cy = Cycle(args.config, seed=rank, layers=args.layers, device=dev)
@@ -453,7 +455,8 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": config_dict(w, k, cy.layers, {"parallelism": f"dp{world} (independent batches per GPU)",
-                                                 "pdl": args.pdl, "fused_merge": args.fused_merge}),
+                                                 "pdl": args.pdl, "fused_merge": args.fused_merge,
+                                                 "ctas_per_sm": args.ctas_per_sm, "early_kv": args.early_kv}),
         "clocks": clocks.summary(),
         "e2e": {"value": world * w.batch * k / (e2e_ms * 1e-3), "unit": "tokens/s",
                 "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -213,11 +213,26 @@ kap_status kap_verify_attn(
  * KAP_ERR_TIMEOUT or KAP_ERR_DEVICE_INDEX), clearing it. */
 kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);
 
-/* Tuning knobs of the attention launches, process-wide: `use_pdl` != 0 launches with programmatic
- * stream serialisation (the next kernel's prologue overlaps the previous kernel's tail);
- * `fused_merge` != 0 lets the last split of a (sequence, KV head) to finish merge the splits
- * inside the split kernel instead of launching the separate merge pass.  Negative = keep. */
-kap_status kap_set_launch_options(int32_t use_pdl, int32_t fused_merge);
+/* Tuning knobs of the attention launches, process-wide; a negative value keeps the setting.
+ *   use_pdl      != 0 (default): launch with programmatic stream serialisation, so that a kernel's
+ *                prologue overlaps the tail of the previous kernel on the stream when that kernel
+ *                releases its dependents early (this library's kernels do; ordinary kernels
+ *                release them only when they complete, which changes nothing).  Before the
+ *                previous kernel has completed an attention kernel reads only static metadata:
+ *                the work list, the page lists and q_indptr.  Those arrays must therefore be
+ *                final before the previous kernel was launched.
+ *   early_kv     != 0 (default; needs use_pdl): in that window the kernel also reads ctx_len and
+ *                starts loading KV pages that hold only tokens older than the query rows' own
+ *                (t < ctx_len - n_q) - pages written in earlier decoding steps.  ctx_len and those
+ *                pages must then be final before the previous kernel was launched; Q, the pages
+ *                holding the rows' own tokens, out and lse may still be written by it.
+ *   fused_merge  != 0: the last split of a (sequence, KV head) to finish merges the splits inside
+ *                the split kernel instead of launching the separate merge pass (default 0).
+ *   ctas_per_sm  resident CTAs per SM the scheduler fills in one wave; 0 = as many as fit.
+ *                Takes effect at the next kap_schedule.
+ * The paper has no counterpart for these. */
+kap_status kap_set_launch_options(int32_t use_pdl, int32_t fused_merge, int32_t ctas_per_sm,
+                                  int32_t early_kv);
 
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t kap_launch_count(void);

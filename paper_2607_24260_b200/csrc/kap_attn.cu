@@ -3,13 +3,13 @@
 // KAP paper, plus the log-sum-exp merge of the splits.
 //
 // One CTA = one work item = a contiguous slice of one sequence's page list for one KV head.
-//   * a producer warp (one elected lane) walks the slice's physical page ids and issues TMA tensor
-//     loads (cp.async.bulk.tensor, 128-byte swizzle) of each page's K and V rows for this KV head
-//     into a ring of shared-memory stages, completion tracked by mbarriers;
-//   * four consumer warps each own one 16-row tile of query rows (rows = n_q * G: the G query
-//     heads of the KV head's group times the n_q query tokens, so every K/V byte is read from HBM
-//     once and shared by all of them), compute S = Q K^T and O += P V with bf16 mma.sync tiles and
-//     fp32 accumulators, and keep a base-2 online softmax per row in registers;
+//   * each page's K and V rows for this KV head arrive by TMA tensor loads (cp.async.bulk.tensor,
+//     128-byte swizzle) in a ring of shared-memory page slots, completion tracked by mbarriers;
+//     one elected lane per warp group keeps the group's slots refilled;
+//   * four warps each own one 16-row tile of query rows (rows = n_q * G: the G query heads of
+//     the KV head's group times the n_q query tokens, so every K/V byte is read from HBM once and
+//     shared by all of them), compute S = Q K^T and O += P V with bf16 mma.sync tiles and fp32
+//     accumulators, and keep a base-2 online softmax per row in registers;
 //   * the warps' states are combined through shared memory and the CTA writes either the final
 //     bf16 output (single split) or an un-normalised fp32 partial (m, l, O) for the merge pass.
 // The proposal path is the n_q = 1 case of the same kernel; the causal rule "row j sees tokens
@@ -21,6 +21,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstring>
 #include <mutex>
@@ -37,32 +38,31 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
                           int32_t* max_chunk_out, int32_t* row_tiles_out);
 
 // ------------------------------------------------------------------------------ kernel geometry
-constexpr int kConsumerWarps = 4;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;       // + the producer warp
-constexpr int kStagePages = 4;                            // pages per pipeline stage
-constexpr int kStages = 3;
+constexpr int kWarps = 4;
+constexpr int kThreads = kWarps * 32;
+constexpr int kSlots = 8;                                 // page slots in the shared-memory ring
 constexpr int kHalfTileBytes = kPageSize * 128;           // 16 tokens x 64 bf16 = 2048 B
 constexpr int kTileBytes = 2 * kHalfTileBytes;            // K (or V) of one page and head: 4096 B
 constexpr int kPageHeadBytes = 2 * kTileBytes;            // K + V: 8192 B
-constexpr int kStageBytes = kStagePages * kPageHeadBytes; // 32 KiB
+constexpr int kRingBytes = kSlots * kPageHeadBytes;       // 64 KiB
 constexpr int kMaxChunk = 512;                            // page ids a CTA can hold
 constexpr int kScratchStride = kHeadDim + 8;              // floats per scratch row (bank spread)
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;         // per-CTA deadline for all waits
 
-struct SmemTail {                                         // what follows the tile ring
+struct SmemTail {                                         // what follows the ring
     int32_t phys[kMaxChunk];
     int32_t logical[kMaxChunk];
-    unsigned long long full[kStages];
-    unsigned long long empty[kStages];
-    float m[kConsumerWarps][kRowTile];
-    float l[kConsumerWarps][kRowTile];
+    unsigned long long full[kSlots];
+    unsigned long long empty[kSlots];
+    float m[kWarps][kRowTile];
+    float l[kWarps][kRowTile];
     int32_t is_last;
     int32_t timed_out;
 };
-constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(SmemTail) + 1024;  // + alignment slack
+constexpr int kSmemBytes = kRingBytes + (int)sizeof(SmemTail) + 1024;   // + alignment slack
 
-static_assert(kConsumerWarps * kRowTile * kScratchStride * 4 <= kStages * kStageBytes,
-              "warp-combine scratch must fit in the tile ring");
+static_assert(kWarps * kRowTile * kScratchStride * 4 <= kRingBytes,
+              "warp-combine scratch must fit in the ring");
 
 struct AttnParams {
     const __nv_bfloat16* q;          // [rows, Hq, d]
@@ -81,9 +81,19 @@ struct AttnParams {
     int32_t* status;
     long long num_pool_pages;
     int32_t Hq, Hkv, G, rows_cap;
-    int32_t fused_merge;
+    int32_t fused_merge, early_kv;
     float scale_log2;                // sm_scale * log2(e)
+#ifdef KAP_TRACE
+    unsigned long long* trace;       // [8192 records][8] timestamps of this launch (debug builds)
+#endif
 };
+
+#ifdef KAP_TRACE
+#define KAP_TRACE_POINT(rec, slot) \
+    do { if (p.trace && threadIdx.x == 0) p.trace[(size_t)(rec) * 8 + (slot)] = global_ns(); } while (0)
+#else
+#define KAP_TRACE_POINT(rec, slot) do { } while (0)
+#endif
 
 // ------------------------------------------------------------------------------- PTX primitives
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -161,29 +171,26 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
-__device__ __forceinline__ void consumer_sync() {           // the 128 consumer threads only
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+// Programmatic dependent launch: let the next kernel on the stream start its prologue now ...
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
+// ... and wait for the previous kernel on the stream to have completed (memory visible).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ------------------------------------------------------------------ merging partial softmax states
-// Combine `n` states (m_i in log2 units, l_i, O_i[4]) read through the accessors into one.
-// Used for warps inside a CTA and for the splits of a (sequence, KV head).
+// (m in log2 units, l, O[4 columns]) states combine as
+//     M = max m_i,  l = sum 2^(m_i - M) l_i,  O = sum 2^(m_i - M) O_i.
 struct Merged { float m, l; float4 o; };
 
-template <typename GetM, typename GetL, typename GetO>
-__device__ __forceinline__ Merged merge_states(int n, GetM get_m, GetL get_l, GetO get_o) {
-    float mx = -INFINITY;
-    for (int i = 0; i < n; ++i) mx = fmaxf(mx, get_m(i));
-    const float mu = (mx == -INFINITY) ? 0.f : mx;
-    Merged r; r.m = mx; r.l = 0.f; r.o = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i = 0; i < n; ++i) {
-        const float w = ex2(get_m(i) - mu);
-        const float4 o = get_o(i);
-        r.l = fmaf(w, get_l(i), r.l);
-        r.o.x = fmaf(w, o.x, r.o.x); r.o.y = fmaf(w, o.y, r.o.y);
-        r.o.z = fmaf(w, o.z, r.o.z); r.o.w = fmaf(w, o.w, r.o.w);
-    }
-    return r;
+__device__ __forceinline__ void merge_into(Merged& r, float m, float l, const float4& o) {
+    const float mn = fmaxf(r.m, m);
+    const float mu = (mn == -INFINITY) ? 0.f : mn;
+    const float a = ex2(r.m - mu), b = ex2(m - mu);
+    r.l = r.l * a + l * b;
+    r.o.x = r.o.x * a + o.x * b; r.o.y = r.o.y * a + o.y * b;
+    r.o.z = r.o.z * a + o.z * b; r.o.w = r.o.w * a + o.w * b;
+    r.m = mn;
 }
 
 // normalise, round to bf16 and store 4 consecutive outputs; lse in natural log
@@ -199,63 +206,72 @@ __device__ __forceinline__ void store_final(const AttnParams& p, int64_t q_row, 
 }
 
 // Merge the splits of one group and write its final rows.  `tid` / `nthreads` enumerate the
-// calling threads; each handles (row, 4-column) cells.
+// calling threads; each handles (row, 4-column) cells.  The partials are read in batches of
+// independent loads so that a cell costs one memory round trip per batch.
 __device__ __forceinline__ void merge_group_splits(const AttnParams& p, const MergeGroup& g,
-                                                   int tid, int nthreads) {
+                                                   int64_t q_row0, int tid, int nthreads) {
+    constexpr int kBatch = 8;
     const int rows = g.n_q * p.G;
-    const int64_t q_row0 = p.q_indptr ? p.q_indptr[g.seq] : g.seq;
     for (int idx = tid; idx < rows * 32; idx += nthreads) {
         const int R = idx >> 5, c4 = idx & 31;
         const int64_t base = (int64_t)g.first_item * p.rows_cap + R;
         const int64_t stride = p.rows_cap;
-        const float* ml = p.part_ml;
-        const float* po = p.part_o;
-        Merged r = merge_states(
-            g.n_splits,
-            [&](int i) { return __ldcg(ml + (base + i * stride) * 2); },
-            [&](int i) { return __ldcg(ml + (base + i * stride) * 2 + 1); },
-            [&](int i) {
-                return __ldcg(reinterpret_cast<const float4*>(po + (base + i * stride) * kHeadDim) + c4);
-            });
+        Merged r; r.m = -INFINITY; r.l = 0.f; r.o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i0 = 0; i0 < g.n_splits; i0 += kBatch) {
+            float2 ml[kBatch];
+            float4 o[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int i = min(i0 + j, g.n_splits - 1);
+                ml[j] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + i * stride) * 2));
+                o[j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (base + i * stride) * kHeadDim) + c4);
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j)
+                if (i0 + j < g.n_splits) merge_into(r, ml[j].x, ml[j].y, o[j]);
+        }
         store_final(p, q_row0 + R / p.G, g.kv_head * p.G + R % p.G, c4, r);
     }
 }
 
 // ------------------------------------------------------------------------------ the split kernel
-__global__ void __launch_bounds__(kThreads, 2)
+// Shared-memory ring: 8 page slots of 8 KiB (K tile then V tile, each two 64-column halves in the
+// TMA 128-byte swizzle).  With RT row tiles the 4 warps form 4/RT warp groups; page i of the slice
+// belongs to group i mod (4/RT) and is consumed by that group's RT warps (one per row tile).  Each
+// group owns 8/(4/RT) slots as a private ring; lane 0 of the group's first warp refills a slot as
+// soon as all RT warps have released it, so every group always has its whole ring in flight.
+__global__ void __launch_bounds__(kThreads, 3)
 kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     // the 128-byte swizzle pattern repeats every 1024 bytes: tiles must start on that boundary
-    unsigned char* tiles = reinterpret_cast<unsigned char*>(
+    unsigned char* ring = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    SmemTail* tail = reinterpret_cast<SmemTail*>(tiles + kStages * kStageBytes);
+    SmemTail* tail = reinterpret_cast<SmemTail*>(ring + kRingBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_launch_dependents();
+    KAP_TRACE_POINT(blockIdx.x, 0);
 
+    // ---- prologue on static metadata only (work list, page lists, q_indptr): with programmatic
+    // dependent launch it overlaps the tail of the previous kernel on the stream.
+    const WorkItem item = p.items[blockIdx.x];
+    const int n_pages = item.page_end - item.page_begin;
+    const int rows = item.n_q * p.G;                         // valid query rows of this item
+    int RT = (rows + kRowTile - 1) / kRowTile;               // row tiles: 1, 2 or 4
+    if (RT == 3) RT = 4;
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kSlots; ++s) {
             mbar_init(smem_u32(&tail->full[s]), 1);
-            mbar_init(smem_u32(&tail->empty[s]), kConsumerWarps);
+            mbar_init(smem_u32(&tail->empty[s]), RT);
         }
         tail->is_last = 0;
         tail->timed_out = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map) : "memory");
     }
-    // Programmatic dependent launch: everything above overlaps the previous kernel's tail; nothing
-    // below (work list, Q, KV, partials) is touched before the previous kernel has completed.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-    const WorkItem item = p.items[blockIdx.x];
-    const int n_pages = item.page_end - item.page_begin;
-    const int n_iters = (n_pages + kStagePages - 1) / kStagePages;
-    const int L = p.ctx_len[item.seq];
     const int64_t list0 = (int64_t)p.list_indptr[item.seq] + item.page_begin;
     const int64_t list_end = p.list_indptr[item.seq + 1];
-    const uint64_t deadline = global_ns() + kWaitBudgetNs;
-
-    // page ids of the slice -> shared memory (they gate every TMA address)
+    const int64_t q_row0 = p.q_indptr ? p.q_indptr[item.seq] : item.seq;
     for (int i = tid; i < n_pages; i += kThreads) {
         int32_t ph = 0;
         bool ok = (list0 + i) < list_end;
@@ -268,46 +284,56 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         tail->logical[i] = p.logical_pages && ok ? p.logical_pages[list0 + i] : item.page_begin + i;
     }
     __syncthreads();
+    KAP_TRACE_POINT(blockIdx.x, 1);
 
-    if (warp == kConsumerWarps) {
-        // ------------------------------------------------------------------ producer warp
-        if (lane == 0) {
-            uint64_t policy;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-            const int rows_per_page = 2 * p.Hkv * kPageSize;
-            const int v_row_off = p.Hkv * kPageSize;
-            for (int it = 0; it < n_iters; ++it) {
-                const int s = it % kStages;
-                if (it >= kStages)
-                    mbar_wait(smem_u32(&tail->empty[s]), ((it / kStages) - 1) & 1, deadline,
-                              &tail->timed_out);
-                const int np = min(kStagePages, n_pages - it * kStagePages);
-                const uint32_t bar = smem_u32(&tail->full[s]);
-                mbar_expect_tx(bar, np * kPageHeadBytes);
-                for (int ps = 0; ps < np; ++ps) {
-                    const int y = tail->phys[it * kStagePages + ps] * rows_per_page
-                                  + item.kv_head * kPageSize;
-                    const uint32_t dst = smem_u32(tiles + s * kStageBytes + ps * kPageHeadBytes);
-                    tma_load_2d(dst, &kv_map, 0, y, bar, policy);
-                    tma_load_2d(dst + kHalfTileBytes, &kv_map, 64, y, bar, policy);
-                    tma_load_2d(dst + kTileBytes, &kv_map, 0, y + v_row_off, bar, policy);
-                    tma_load_2d(dst + kTileBytes + kHalfTileBytes, &kv_map, 64, y + v_row_off, bar,
-                                policy);
-                }
+    const int n_groups = kWarps / RT;                        // warp groups
+    const int depth = kSlots / n_groups;                     // ring slots per group
+    const int grp = warp / RT, rt = warp % RT;
+    const int n_mine = grp < n_pages ? (n_pages - grp + n_groups - 1) / n_groups : 0;
+    const bool producer = (rt == 0) && (lane == 0);
+    const int rows_per_page = 2 * p.Hkv * kPageSize;
+    const int v_row_off = p.Hkv * kPageSize;
+    uint64_t policy = 0;
+    if (producer) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+
+    // issue the loads of this group's i-th page into ring slot grp * depth + i % depth
+    auto issue = [&](int i) {
+        const int s = grp * depth + i % depth;
+        const uint32_t bar = smem_u32(&tail->full[s]);
+        const int y = tail->phys[grp + i * n_groups] * rows_per_page + item.kv_head * kPageSize;
+        const uint32_t dst = smem_u32(ring + s * kPageHeadBytes);
+        mbar_expect_tx(bar, kPageHeadBytes);
+        tma_load_2d(dst, &kv_map, 0, y, bar, policy);
+        tma_load_2d(dst + kHalfTileBytes, &kv_map, 64, y, bar, policy);
+        tma_load_2d(dst + kTileBytes, &kv_map, 0, y + v_row_off, bar, policy);
+        tma_load_2d(dst + kTileBytes + kHalfTileBytes, &kv_map, 64, y + v_row_off, bar, policy);
+    };
+    // Early KV prefetch: pages that hold only tokens older than the query rows' own tokens
+    // (t < L - n_q) were written in earlier steps, so their loads may start before the previous
+    // kernel on the stream has completed.  Pages holding the rows' own tokens, Q and the partial
+    // buffers wait for it.  (ctx_len must then be final before the previous kernel was launched.)
+    const int first = min(depth, n_mine);
+    int issued = 0, L = 0;
+    if (p.early_kv) {
+        L = p.ctx_len[item.seq];
+        if (producer) {
+            const int fresh_from = L - item.n_q;
+            while (issued < first &&
+                   tail->logical[grp + issued * n_groups] * kPageSize + kPageSize - 1 < fresh_from) {
+                issue(issued);
+                ++issued;
             }
         }
-        return;      // every load it issued is awaited by the consumers before they finish
     }
+    // ---- nothing else produced by earlier kernels (Q, fresh KV, partial buffers) is touched above
+    pdl_wait();
+    KAP_TRACE_POINT(blockIdx.x, 2);
+    if (producer)
+        for (; issued < first; ++issued) issue(issued);
+    if (!p.early_kv) L = p.ctx_len[item.seq];
+    const uint64_t deadline = global_ns() + kWaitBudgetNs;
 
-    // ---------------------------------------------------------------------- consumer warps
     const int gid = lane >> 2, tid4 = lane & 3;
-    const int rows = item.n_q * p.G;                         // valid query rows of this item
-    int RT = (rows + kRowTile - 1) / kRowTile;               // row tiles: 1, 2 or 4
-    if (RT == 3) RT = 4;
-    const int rt = warp % RT;                                // this warp's row tile
-    const int ps0 = warp / RT, ps_step = kConsumerWarps / RT;
-    const int64_t q_row0 = p.q_indptr ? p.q_indptr[item.seq] : item.seq;
-
     // Q fragments (A operand, 16 rows x 128) straight from global memory, zero for padding rows.
     // Row R of the item = query token R / G, head R % G of the group.
     uint32_t qf[8][4];
@@ -341,92 +367,97 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     const int k_tok = ((lm >> 1) << 3) + lr, k_cbit = lm & 1;   // K: matrices (n-tile, k-half)
     const int v_tok = ((lm & 1) << 3) + lr, v_cbit = lm >> 1;   // V^T: matrices (k-half, n-tile)
 
-    for (int it = 0; it < n_iters; ++it) {
-        const int s = it % kStages;
-        mbar_wait(smem_u32(&tail->full[s]), (it / kStages) & 1, deadline, &tail->timed_out);
-        const int np = min(kStagePages, n_pages - it * kStagePages);
-        for (int ps = ps0; ps < np; ps += ps_step) {
-            const uint32_t kb = smem_u32(tiles + s * kStageBytes + ps * kPageHeadBytes);
-            const uint32_t vb = kb + kTileBytes;
-            const int tok0 = tail->logical[it * kStagePages + ps] * kPageSize;
+    for (int i = 0; i < n_mine; ++i) {
+        const int s = grp * depth + i % depth;
+        const uint32_t parity = (i / depth) & 1;
+        mbar_wait(smem_u32(&tail->full[s]), parity, deadline, &tail->timed_out);
+        if (i == 0) KAP_TRACE_POINT(blockIdx.x, 3);
+        const uint32_t kb = smem_u32(ring + s * kPageHeadBytes);
+        const uint32_t vb = kb + kTileBytes;
+        const int tok0 = tail->logical[grp + i * n_groups] * kPageSize;
 
-            // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
-            float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
+        float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                uint32_t b0, b1, b2, b3;
-                ldsm_x4(kb + (ks >> 2) * kHalfTileBytes + k_tok * 128
-                           + ((((ks & 3) * 2 + k_cbit) ^ lr) << 4), b0, b1, b2, b3);
-                mma_bf16(sacc[0], qf[ks], b0, b1);
-                mma_bf16(sacc[1], qf[ks], b2, b3);
-            }
-            if (tok0 + kPageSize - 1 > full_vis_limit) {
-                // page reaches into the causal / tail region: mask per element
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4(kb + (ks >> 2) * kHalfTileBytes + k_tok * 128
+                       + ((((ks & 3) * 2 + k_cbit) ^ lr) << 4), b0, b1, b2, b3);
+            mma_bf16(sacc[0], qf[ks], b0, b1);
+            mma_bf16(sacc[1], qf[ks], b2, b3);
+        }
+        if (tok0 + kPageSize - 1 > full_vis_limit) {
+            // page reaches into the causal / tail region: mask per element
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt)
+            for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int t = tok0 + nt * 8 + tid4 * 2 + (e & 1);
-                        if (t > pos_row[e >> 1]) sacc[nt][e] = -INFINITY;
-                    }
-                // value rows past the end of the context may hold anything (even NaN): zero them
-                const int first_bad = L - tok0;
-                if (first_bad < kPageSize) {
-                    if (lane < 16) {
-                        for (int r = max(first_bad, 0); r < kPageSize; ++r)
-                            *reinterpret_cast<uint4*>(tiles + s * kStageBytes + ps * kPageHeadBytes
-                                                      + kTileBytes + (lane >> 3) * kHalfTileBytes
-                                                      + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
+                for (int e = 0; e < 4; ++e) {
+                    const int t = tok0 + nt * 8 + tid4 * 2 + (e & 1);
+                    if (t > pos_row[e >> 1]) sacc[nt][e] = -INFINITY;
                 }
-            }
-            // online softmax (base 2): rows gid (e = 0,1) and gid + 8 (e = 2,3)
-            float mx[2];
-            mx[0] = fmaxf(fmaxf(sacc[0][0], sacc[0][1]), fmaxf(sacc[1][0], sacc[1][1]));
-            mx[1] = fmaxf(fmaxf(sacc[0][2], sacc[0][3]), fmaxf(sacc[1][2], sacc[1][3]));
-            float corr[2], mu[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
-                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-                const float mn = fmaxf(m_run[h], mx[h] * sc);
-                mu[h] = (mn == -INFINITY) ? 0.f : mn;
-                corr[h] = ex2(m_run[h] - mu[h]);
-                m_run[h] = mn;
-            }
-            uint32_t pa[4];      // P as the A operand of P V (rows gid / gid+8, tokens 0-7 / 8-15)
-            pa[0] = pack_bf16(ex2(fmaf(sacc[0][0], sc, -mu[0])), ex2(fmaf(sacc[0][1], sc, -mu[0])));
-            pa[1] = pack_bf16(ex2(fmaf(sacc[0][2], sc, -mu[1])), ex2(fmaf(sacc[0][3], sc, -mu[1])));
-            pa[2] = pack_bf16(ex2(fmaf(sacc[1][0], sc, -mu[0])), ex2(fmaf(sacc[1][1], sc, -mu[0])));
-            pa[3] = pack_bf16(ex2(fmaf(sacc[1][2], sc, -mu[1])), ex2(fmaf(sacc[1][3], sc, -mu[1])));
-            // the row sums use the rounded weights, so out = sum(p v) / sum(p) is a true average
-            l_run[0] = fmaf(l_run[0], corr[0],
-                            (bf16_lo(pa[0]) + bf16_hi(pa[0])) + (bf16_lo(pa[2]) + bf16_hi(pa[2])));
-            l_run[1] = fmaf(l_run[1], corr[1],
-                            (bf16_lo(pa[1]) + bf16_hi(pa[1])) + (bf16_lo(pa[3]) + bf16_hi(pa[3])));
-            if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    o[i][0] *= corr[0]; o[i][1] *= corr[0];
-                    o[i][2] *= corr[1]; o[i][3] *= corr[1];
+            // value rows past the end of the context may hold anything (even NaN): zero them
+            const int first_bad = L - tok0;
+            if (first_bad < kPageSize) {
+                if (lane < 16) {
+                    for (int r = max(first_bad, 0); r < kPageSize; ++r)
+                        *reinterpret_cast<uint4*>(ring + s * kPageHeadBytes + kTileBytes
+                                                  + (lane >> 3) * kHalfTileBytes + r * 128
+                                                  + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
                 }
-            }
-            // O += P V   (16 n-tiles of 8 output columns, two per ldmatrix)
-#pragma unroll
-            for (int n2 = 0; n2 < 8; ++n2) {
-                uint32_t v0, v1, v2, v3;
-                ldsm_x4_t(vb + (n2 >> 2) * kHalfTileBytes + v_tok * 128
-                             + ((((n2 & 3) * 2 + v_cbit) ^ lr) << 4), v0, v1, v2, v3);
-                mma_bf16(o[2 * n2], pa, v0, v1);
-                mma_bf16(o[2 * n2 + 1], pa, v2, v3);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
             }
         }
+        // online softmax (base 2): rows gid (e = 0,1) and gid + 8 (e = 2,3)
+        float mx[2];
+        mx[0] = fmaxf(fmaxf(sacc[0][0], sacc[0][1]), fmaxf(sacc[1][0], sacc[1][1]));
+        mx[1] = fmaxf(fmaxf(sacc[0][2], sacc[0][3]), fmaxf(sacc[1][2], sacc[1][3]));
+        float corr[2], mu[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+            const float mn = fmaxf(m_run[h], mx[h] * sc);
+            mu[h] = (mn == -INFINITY) ? 0.f : mn;
+            corr[h] = ex2(m_run[h] - mu[h]);
+            m_run[h] = mn;
+        }
+        uint32_t pa[4];      // P as the A operand of P V (rows gid / gid+8, tokens 0-7 / 8-15)
+        pa[0] = pack_bf16(ex2(fmaf(sacc[0][0], sc, -mu[0])), ex2(fmaf(sacc[0][1], sc, -mu[0])));
+        pa[1] = pack_bf16(ex2(fmaf(sacc[0][2], sc, -mu[1])), ex2(fmaf(sacc[0][3], sc, -mu[1])));
+        pa[2] = pack_bf16(ex2(fmaf(sacc[1][0], sc, -mu[0])), ex2(fmaf(sacc[1][1], sc, -mu[0])));
+        pa[3] = pack_bf16(ex2(fmaf(sacc[1][2], sc, -mu[1])), ex2(fmaf(sacc[1][3], sc, -mu[1])));
+        // the row sums use the rounded weights, so out = sum(p v) / sum(p) is a true average
+        l_run[0] = fmaf(l_run[0], corr[0],
+                        (bf16_lo(pa[0]) + bf16_hi(pa[0])) + (bf16_lo(pa[2]) + bf16_hi(pa[2])));
+        l_run[1] = fmaf(l_run[1], corr[1],
+                        (bf16_lo(pa[1]) + bf16_hi(pa[1])) + (bf16_lo(pa[3]) + bf16_hi(pa[3])));
+        if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+            for (int n = 0; n < 16; ++n) {
+                o[n][0] *= corr[0]; o[n][1] *= corr[0];
+                o[n][2] *= corr[1]; o[n][3] *= corr[1];
+            }
+        }
+        // O += P V   (16 n-tiles of 8 output columns, two per ldmatrix)
+#pragma unroll
+        for (int n2 = 0; n2 < 8; ++n2) {
+            uint32_t v0, v1, v2, v3;
+            ldsm_x4_t(vb + (n2 >> 2) * kHalfTileBytes + v_tok * 128
+                         + ((((n2 & 3) * 2 + v_cbit) ^ lr) << 4), v0, v1, v2, v3);
+            mma_bf16(o[2 * n2], pa, v0, v1);
+            mma_bf16(o[2 * n2 + 1], pa, v2, v3);
+        }
+        // release the slot; the group's producer lane refills it once all RT warps have
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&tail->empty[s]));
+        if (producer && i + depth < n_mine) {
+            mbar_wait(smem_u32(&tail->empty[s]), parity, deadline, &tail->timed_out);
+            issue(i + depth);
+        }
     }
     if (lane == 0 && tail->timed_out) atomicOr(p.status, 1 << KAP_ERR_TIMEOUT);
+    KAP_TRACE_POINT(blockIdx.x, 4);
 
     // ------------------------------------------------ combine the four warps' states, write out
 #pragma unroll
@@ -434,35 +465,32 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 1);
         l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 2);
     }
-    consumer_sync();                                   // all tile reads done: the ring is scratch now
-    float* scratch = reinterpret_cast<float*>(tiles) + warp * (kRowTile * kScratchStride);
+    __syncthreads();                                   // all tile reads done: the ring is scratch now
+    float* scratch = reinterpret_cast<float*>(ring) + warp * (kRowTile * kScratchStride);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        *reinterpret_cast<float2*>(scratch + gid * kScratchStride + i * 8 + tid4 * 2) =
-            make_float2(o[i][0], o[i][1]);
-        *reinterpret_cast<float2*>(scratch + (gid + 8) * kScratchStride + i * 8 + tid4 * 2) =
-            make_float2(o[i][2], o[i][3]);
+    for (int n = 0; n < 16; ++n) {
+        *reinterpret_cast<float2*>(scratch + gid * kScratchStride + n * 8 + tid4 * 2) =
+            make_float2(o[n][0], o[n][1]);
+        *reinterpret_cast<float2*>(scratch + (gid + 8) * kScratchStride + n * 8 + tid4 * 2) =
+            make_float2(o[n][2], o[n][3]);
     }
     if (tid4 == 0) {
         tail->m[warp][gid] = m_run[0];     tail->l[warp][gid] = l_run[0];
         tail->m[warp][gid + 8] = m_run[1]; tail->l[warp][gid + 8] = l_run[1];
     }
-    consumer_sync();
+    __syncthreads();
 
-    const float* all = reinterpret_cast<const float*>(tiles);
-    const int n_same = kConsumerWarps / RT;            // warps that share a row tile
+    const float* all = reinterpret_cast<const float*>(ring);
     const bool single = item.n_splits == 1;
-    for (int idx = tid; idx < rows * 32; idx += kConsumerWarps * 32) {
+    for (int idx = tid; idx < rows * 32; idx += kThreads) {
         const int R = idx >> 5, c4 = idx & 31;
         const int t = R / kRowTile, r = R % kRowTile;
-        Merged res = merge_states(
-            n_same,
-            [&](int i) { return tail->m[t + i * RT][r]; },
-            [&](int i) { return tail->l[t + i * RT][r]; },
-            [&](int i) {
-                return *reinterpret_cast<const float4*>(
-                    all + ((t + i * RT) * kRowTile + r) * kScratchStride + c4 * 4);
-            });
+        Merged res; res.m = -INFINITY; res.l = 0.f; res.o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int g = 0; g < n_groups; ++g) {            // warps g * RT + t hold row tile t
+            const int w = g * RT + t;
+            merge_into(res, tail->m[w][r], tail->l[w][r],
+                       *reinterpret_cast<const float4*>(all + (w * kRowTile + r) * kScratchStride + c4 * 4));
+        }
         if (single) {
             store_final(p, q_row0 + R / p.G, item.kv_head * p.G + R % p.G, c4, res);
         } else {
@@ -471,21 +499,30 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             if (c4 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(res.m, res.l);
         }
     }
+    KAP_TRACE_POINT(blockIdx.x, 5);
+#ifdef KAP_TRACE
+    if (p.trace && tid == 0) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        p.trace[(size_t)blockIdx.x * 8 + 7] = smid;
+    }
+#endif
     if (single || !p.fused_merge) return;
 
     // Fused merge: the last split of the group to arrive combines all of them.
     __threadfence();
-    consumer_sync();
+    __syncthreads();
     if (tid == 0) {
         const int prev = atomicAdd(p.counters + item.group, 1);
         const int last = prev == item.n_splits - 1;
         if (last) p.counters[item.group] = 0;           // leave the counter clean for the next launch
         tail->is_last = last;
     }
-    consumer_sync();
+    __syncthreads();
     if (!tail->is_last) return;
     __threadfence();
-    merge_group_splits(p, p.groups[item.group], tid, kConsumerWarps * 32);
+    merge_group_splits(p, p.groups[item.group], q_row0, tid, kThreads);
+    KAP_TRACE_POINT(blockIdx.x, 6);
 }
 
 // -------------------------------------------------------------------- the separate merge kernel
@@ -493,9 +530,14 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
 __global__ void __launch_bounds__(128)
 kap_attn_merge_kernel(const AttnParams p, const MergeGroup* merge_groups)
 {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    merge_group_splits(p, merge_groups[blockIdx.x], threadIdx.x, blockDim.x);
+    pdl_launch_dependents();
+    KAP_TRACE_POINT(4096 + blockIdx.x, 0);
+    const MergeGroup g = merge_groups[blockIdx.x];          // static metadata: before the wait
+    const int64_t q_row0 = p.q_indptr ? p.q_indptr[g.seq] : g.seq;
+    pdl_wait();
+    KAP_TRACE_POINT(4096 + blockIdx.x, 2);
+    merge_group_splits(p, g, q_row0, threadIdx.x, blockDim.x);
+    KAP_TRACE_POINT(4096 + blockIdx.x, 5);
 }
 
 // ================================================================================= host side
@@ -504,6 +546,8 @@ namespace {
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_use_pdl{1};
 std::atomic<int> g_fused_merge{0};
+std::atomic<int> g_early_kv{1};
+std::atomic<int> g_ctas_per_sm{0};       // 0 = as many as fit (occupancy)
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -561,6 +605,11 @@ kap_status get_tensor_map(kap_workspace* ws, const void* pool, int64_t pages, in
     return KAP_OK;
 }
 
+#ifdef KAP_TRACE
+unsigned long long* g_trace = nullptr;      // [g_trace_cap launches][8192][8]
+int g_trace_cap = 0, g_trace_next = 0;
+#endif
+
 std::once_flag g_attr_once;
 cudaError_t g_attr_err = cudaSuccess;
 
@@ -579,6 +628,10 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
 
     AttnParams p = p_in;
     p.fused_merge = g_fused_merge.load() ? 1 : 0;
+    p.early_kv = (g_use_pdl.load() && g_early_kv.load()) ? 1 : 0;
+#ifdef KAP_TRACE
+    p.trace = (g_trace && g_trace_next < g_trace_cap) ? g_trace + (size_t)(g_trace_next++) * 8192 * 8 : nullptr;
+#endif
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -672,6 +725,7 @@ extern "C" kap_status kap_workspace_create(kap_workspace** out, int32_t device, 
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kap_attn_split_kernel, kThreads,
                                                       kSmemBytes) != cudaSuccess || per_sm < 1)
         per_sm = 1;
+    ws->occupancy = per_sm;
     ws->ctas_per_wave = per_sm * ws->sm_count;
     *out = ws;
     return KAP_OK;
@@ -696,6 +750,8 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     std::vector<WorkItem> items;
     std::vector<MergeGroup> groups;
     int32_t max_chunk = 0, row_tiles = 1;
+    const int want = g_ctas_per_sm.load();
+    ws->ctas_per_wave = (want > 0 ? std::min(want, ws->occupancy) : ws->occupancy) * ws->sm_count;
     kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, ws->ctas_per_wave,
                                    max_chunk_pages, ws->max_items, ws->max_rows, items, groups,
                                    &max_chunk, &row_tiles);
@@ -801,10 +857,29 @@ extern "C" kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream) 
     return KAP_OK;
 }
 
-extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t fused_merge) {
+extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t fused_merge, int32_t ctas_per_sm,
+                                             int32_t early_kv) {
+    if (early_kv >= 0) g_early_kv.store(early_kv ? 1 : 0);
     if (use_pdl >= 0) g_use_pdl.store(use_pdl ? 1 : 0);
     if (fused_merge >= 0) g_fused_merge.store(fused_merge ? 1 : 0);
+    if (ctas_per_sm >= 0) g_ctas_per_sm.store(ctas_per_sm);
     return KAP_OK;
 }
 
 extern "C" int64_t kap_launch_count(void) { return g_launches.load(); }
+
+#ifdef KAP_TRACE
+// Debug builds only: device-side timestamps per CTA.  Launch l writes records [l][cta][8].
+extern "C" int kap_debug_trace_begin(int launches) {
+    if (g_trace) cudaFree(g_trace);
+    g_trace = nullptr;
+    g_trace_cap = launches; g_trace_next = 0;
+    if (cudaMalloc((void**)&g_trace, (size_t)launches * 8192 * 8 * 8) != cudaSuccess) return 1;
+    cudaMemset(g_trace, 0, (size_t)launches * 8192 * 8 * 8);
+    return 0;
+}
+extern "C" int kap_debug_trace_read(unsigned long long* host, int launches) {
+    cudaDeviceSynchronize();
+    return cudaMemcpy(host, g_trace, (size_t)launches * 8192 * 8 * 8, cudaMemcpyDeviceToHost) != cudaSuccess;
+}
+#endif

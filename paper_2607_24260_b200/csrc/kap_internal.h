@@ -43,7 +43,7 @@ struct MergeGroup {
 struct kap_workspace {
     int32_t device = 0;
     int32_t max_items = 0, max_rows = 0, max_batch = 0;
-    int32_t sm_count = 0;
+    int32_t sm_count = 0, occupancy = 1;
     // last schedule
     int32_t batch = 0, n_items = 0, n_groups = 0, n_merge_groups = 0, max_chunk = 0;
     int32_t ctas_per_wave = 0, row_tiles = 1, num_q_heads = 0, num_kv_heads = 0;

@@ -36,7 +36,7 @@ SIGNATURES = {
     "kap_verify_attn": (C.c_int, [_vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_int32, C.c_int32,
                                   C.c_int32, C.c_int32, C.c_int32, C.c_float, _vp, _vp, _vp, _vp]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
-    "kap_set_launch_options": (C.c_int, [C.c_int32, C.c_int32]),
+    "kap_set_launch_options": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
     "kap_launch_count": (C.c_int64, []),
     "kap_last_error": (C.c_char_p, []),
     "kap_version": (C.c_char_p, []),
@@ -87,8 +87,10 @@ def launch_count() -> int:
     return int(lib().kap_launch_count())
 
 
-def set_launch_options(use_pdl: int = -1, fused_merge: int = -1):
-    _check(lib().kap_set_launch_options(int(use_pdl), int(fused_merge)))
+def set_launch_options(use_pdl: int = -1, fused_merge: int = -1, ctas_per_sm: int = -1,
+                       early_kv: int = -1):
+    _check(lib().kap_set_launch_options(int(use_pdl), int(fused_merge), int(ctas_per_sm),
+                                        int(early_kv)))
 
 
 # ------------------------------------------------------------------------------- kap_compile_plan

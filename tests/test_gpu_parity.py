@@ -286,9 +286,9 @@ def test_split_and_launch_option_invariance():
     ref = gu.oracle_decode(qd, pool_bits, plan, w.ctx_len)
     one_split = gu.run_decode(qd, pool, plan, w.ctx_len, max_chunk_pages=512)
     try:
-        for pdl in (0, 1):
+        for pdl, early in ((0, 0), (1, 0), (1, 1)):
             for fused in (0, 1):
-                kap.set_launch_options(pdl, fused)
+                kap.set_launch_options(pdl, fused, -1, early)
                 for chunk in (0, 1, 7):
                     got = gu.run_decode(qd, pool, plan, w.ctx_len, max_chunk_pages=chunk)
                     _check_pair(got, ref, f"pdl={pdl} fused={fused} chunk={chunk}")
@@ -299,7 +299,7 @@ def test_split_and_launch_option_invariance():
                 _check_pair(got, gu.oracle_verify(q_bits, w.n_q, pool_bits, w.bt_indptr, w.bt_pages, w.ctx_len),
                             f"verify pdl={pdl} fused={fused}")
     finally:
-        kap.set_launch_options(1, 0)
+        kap.set_launch_options(1, 0, -1, 1)
 
 
 def test_repeated_calls_and_workspace_reuse():
@@ -317,7 +317,7 @@ def test_repeated_calls_and_workspace_reuse():
             again = gu.run_decode(qd, pool, plan, w.ctx_len, ws=ws, max_chunk_pages=4)
             np.testing.assert_array_equal(first[0], again[0])
     finally:
-        kap.set_launch_options(1, 0)
+        kap.set_launch_options(1, 0, -1, 1)
         ws.close()
 
 
