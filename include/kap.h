@@ -209,6 +209,58 @@ kap_status kap_verify_attn(
     float* lse,                        /* DEVICE fp32 [sum n_q, Hq] or NULL */
     kap_workspace* ws, void* cuda_stream);
 
+/*
+ * kap_selected_decode_attn_static - the proposal-path attention of kap_selected_decode_attn for
+ * callers that are not allowed to allocate device memory.  (The paper has no counterpart: this is
+ * a packaging of the same computation, not another operation.)
+ *
+ * Who needs it: code that runs inside a host program which reserved the whole GPU up front and
+ * hands out memory through its own pool (an inference server, a plug-in loaded into one), code on
+ * a path where cudaMalloc's implicit device synchronisation is not acceptable, or code that simply
+ * has no safe point at which to create and later destroy a kap_workspace.  Such callers cannot use
+ * the workspace entry points, because kap_workspace_create allocates.
+ *
+ * What is different from kap_selected_decode_attn:
+ *   - no kap_workspace and no kap_schedule.  Every (sequence, KV head) page list is cut into
+ *     `num_splits` near-equal slices by a small kernel on the device; the work list, the merge map,
+ *     the fp32 partial results and the status word live in one array built into the library
+ *     (4 MiB of device memory on every GPU that loads it, held until the process exits).
+ *   - the call makes no cudaMalloc / cudaFree and calls no allocating library routine.  The first
+ *     call on a device looks up the array's device address and sets a kernel attribute (once per
+ *     device, for the device that is current at that moment); make that first call outside any
+ *     stream capture.
+ *   - sizes the array cannot hold are refused: batch * num_kv_heads * num_splits work items need
+ *     about 32 + (Hq/Hkv) * 520 bytes each; beyond 4 MiB in total the call returns
+ *     KAP_ERR_CAPACITY and enqueues nothing (with 32/8 heads: roughly 1900 work items).
+ *   - all calls on a device share the array and it keeps the previous call's contents.  The call
+ *     itself clears the only part that must start at zero (the status word) and rewrites the
+ *     rest before use, so back-to-back calls on ONE stream are fine; calls that may overlap on
+ *     the GPU (different streams, different host threads) race on the array and must be ordered
+ *     by the caller.
+ *   - kernels are launched without programmatic stream serialisation (the work list is produced
+ *     on the device just before it is read).
+ * Results are the same as the workspace entry point's up to the order of the fp32 sums.
+ * device_status (DEVICE int32, may be NULL) receives the kernels' status bits after the call's
+ * kernels: 0, or 1 << KAP_ERR_DEVICE_INDEX / 1 << KAP_ERR_TIMEOUT.
+ * Errors: KAP_ERR_UNSUPPORTED (shape), KAP_ERR_INVALID_ARG (NULL pointer, num_splits < 1,
+ * misaligned pool), KAP_ERR_CAPACITY (see above), KAP_ERR_CUDA.
+ */
+kap_status kap_selected_decode_attn_static(
+    const void* q,                     /* DEVICE bf16 [batch, Hq, d] */
+    const void* kv_pool,               /* DEVICE bf16 [num_pool_pages][2][Hkv][P][d] */
+    int64_t num_pool_pages,
+    const int32_t* plan_indptr,        /* DEVICE [batch+1] */
+    const int32_t* plan_phys_pages,    /* DEVICE */
+    const int32_t* plan_logical_pages, /* DEVICE or NULL */
+    const int32_t* ctx_len,            /* DEVICE [batch] */
+    int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
+    float sm_scale,
+    int32_t num_splits,                /* slices per (sequence, KV head), >= 1 */
+    void* out,                         /* DEVICE bf16 [batch, Hq, d] */
+    float* lse,                        /* DEVICE fp32 [batch, Hq] or NULL */
+    int32_t* device_status,            /* DEVICE int32 or NULL */
+    void* cuda_stream);
+
 /* Synchronises `cuda_stream` and returns the device status word of the workspace (KAP_OK,
  * KAP_ERR_TIMEOUT or KAP_ERR_DEVICE_INDEX), clearing it. */
 kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);

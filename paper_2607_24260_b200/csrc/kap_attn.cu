@@ -883,3 +883,166 @@ extern "C" int kap_debug_trace_read(unsigned long long* host, int launches) {
     return cudaMemcpy(host, g_trace, (size_t)launches * 8192 * 8 * 8, cudaMemcpyDeviceToHost) != cudaSuccess;
 }
 #endif
+
+// ============================================================ allocation-free proposal attention
+// kap_selected_decode_attn_static: the proposal-path attention for callers that must not allocate
+// device memory.  Everything the split-K kernels need beyond the caller's inputs and outputs (the
+// work list, the merge map, the partial results, the status word) lives in one file-scope device
+// array of fixed size, so the call makes no cudaMalloc / cudaFree and needs no kap_workspace.
+namespace kap {
+namespace {
+
+constexpr size_t kStaticScratchBytes = 4u << 20;            // 4 MiB per GPU that loads the library
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices] = {};              // device address of the array, per device
+bool g_static_ready[kMaxDevices] = {};
+
+// Layout of the array for one call: [status word, padded to 256 B][items][groups][part_ml][part_o]
+struct StaticLayout {
+    size_t items_off, groups_off, ml_off, o_off, total;
+};
+StaticLayout static_layout(int64_t n_items, int64_t n_groups, int rows) {
+    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
+    StaticLayout l;
+    l.items_off = 256;
+    l.groups_off = up(l.items_off + sizeof(WorkItem) * (size_t)n_items);
+    l.ml_off = up(l.groups_off + sizeof(MergeGroup) * (size_t)n_groups);
+    l.o_off = up(l.ml_off + sizeof(float) * 2 * (size_t)rows * (size_t)n_items);
+    l.total = up(l.o_off + sizeof(float) * (size_t)kHeadDim * (size_t)rows * (size_t)n_items);
+    return l;
+}
+
+// Every (sequence, KV head) gets exactly `splits` work items of near-equal length (some may be
+// empty when the list is shorter than `splits`); item and partial slot (seq * Hkv + g) * splits + s.
+__global__ void kap_static_build_items_kernel(const int32_t* __restrict__ list_indptr, int batch,
+                                              int hkv, int splits, WorkItem* items,
+                                              MergeGroup* groups) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= batch * hkv * splits) return;
+    const int s = idx % splits, grp = idx / splits, g = grp % hkv, b = grp / hkv;
+    const int n = max(list_indptr[b + 1] - list_indptr[b], 0);
+    const int base = n / splits, rem = n % splits;
+    WorkItem it;
+    it.seq = b; it.kv_head = g;
+    it.page_begin = s * base + min(s, rem);
+    it.page_end = it.page_begin + base + (s < rem ? 1 : 0);
+    it.group = grp; it.split = idx; it.n_splits = splits; it.n_q = 1;
+    items[idx] = it;
+    if (s == 0) {
+        MergeGroup mg;
+        mg.seq = b; mg.kv_head = g; mg.first_item = idx; mg.n_splits = splits; mg.n_q = 1;
+        mg.pad[0] = mg.pad[1] = mg.pad[2] = 0;
+        groups[grp] = mg;
+    }
+}
+
+}  // namespace
+}  // namespace kap
+
+extern "C" kap_status kap_selected_decode_attn_static(
+    const void* q, const void* kv_pool, int64_t num_pool_pages, const int32_t* plan_indptr,
+    const int32_t* plan_phys_pages, const int32_t* plan_logical_pages, const int32_t* ctx_len,
+    int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
+    float sm_scale, int32_t num_splits, void* out, float* lse, int32_t* device_status,
+    void* cuda_stream)
+{
+    if (head_dim != kHeadDim || page_size != kPageSize)
+        return fail(KAP_ERR_UNSUPPORTED, "head_dim %d / page_size %d (supported: 128 / 16)", head_dim, page_size);
+    if (num_q_heads <= 0 || num_kv_heads <= 0 || num_q_heads % num_kv_heads ||
+        kRowTile % (num_q_heads / num_kv_heads))
+        return fail(KAP_ERR_UNSUPPORTED, "head counts %d / %d", num_q_heads, num_kv_heads);
+    if (batch < 0 || num_splits < 1) return fail(KAP_ERR_INVALID_ARG, "batch %d / num_splits %d", batch, num_splits);
+    if (batch == 0) return KAP_OK;
+    if (!q || !kv_pool || !plan_indptr || !plan_phys_pages || !ctx_len || !out || num_pool_pages <= 0)
+        return fail(KAP_ERR_INVALID_ARG, "NULL pointer or empty pool");
+    if (reinterpret_cast<uintptr_t>(kv_pool) & 15) return fail(KAP_ERR_INVALID_ARG, "kv_pool is not 16-byte aligned");
+    const int rows = num_q_heads / num_kv_heads;
+    const int64_t n_groups = (int64_t)batch * num_kv_heads;
+    const int64_t n_items = n_groups * num_splits;
+    const StaticLayout lay = static_layout(n_items, n_groups, rows);
+    if (n_items > (1 << 20) || lay.total > kStaticScratchBytes)
+        return fail(KAP_ERR_CAPACITY,
+                    "batch %d x %d KV heads x %d splits needs %zu bytes of scratch; the built-in array holds %zu "
+                    "(use fewer splits or the workspace entry point)",
+                    batch, num_kv_heads, num_splits, lay.total, kStaticScratchBytes);
+
+    // one-time set-up per device: the array's name is only a host-side handle, the kernels need
+    // its device address on the device that is current now
+    int dev = -1;
+    KAP_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(KAP_ERR_UNSUPPORTED, "device index %d", dev);
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ready[dev]) {
+            void* ptr = nullptr;
+            KAP_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+            KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+            g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+            g_static_ready[dev] = true;
+        }
+    }
+    unsigned char* base = g_static_ptr[dev];
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+    // tensor map on the stack (no cache, no heap)
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return fail(KAP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    const uint64_t pool_rows = (uint64_t)num_pool_pages * 2 * num_kv_heads * kPageSize;
+    if (pool_rows >= (1ull << 31)) return fail(KAP_ERR_UNSUPPORTED, "pool of %lld pages is too large", (long long)num_pool_pages);
+    alignas(64) CUtensorMap map;
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)pool_rows};
+        cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
+        cuuint32_t box[2] = {64, (cuuint32_t)kPageSize};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(kv_pool), dims,
+                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(KAP_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
+    }
+
+    AttnParams p{};
+    p.q = (const __nv_bfloat16*)q; p.q_indptr = nullptr; p.list_indptr = plan_indptr;
+    p.phys_pages = plan_phys_pages; p.logical_pages = plan_logical_pages; p.ctx_len = ctx_len;
+    p.items = reinterpret_cast<const WorkItem*>(base + lay.items_off);
+    p.groups = reinterpret_cast<const MergeGroup*>(base + lay.groups_off);
+    p.part_ml = reinterpret_cast<float*>(base + lay.ml_off);
+    p.part_o = reinterpret_cast<float*>(base + lay.o_off);
+    p.counters = nullptr;
+    p.out = (__nv_bfloat16*)out; p.lse = lse;
+    p.status = reinterpret_cast<int32_t*>(base);
+    p.num_pool_pages = num_pool_pages; p.Hq = num_q_heads; p.Hkv = num_kv_heads; p.G = rows;
+    p.rows_cap = rows; p.fused_merge = 0; p.early_kv = 0;
+    p.scale_log2 = sm_scale * 1.4426950408889634f;
+#ifdef KAP_TRACE
+    p.trace = nullptr;
+#endif
+
+    // the array keeps the previous call's contents: the status word must start at zero; the work
+    // list and merge map are rewritten in full below, and every partial slot that the merge reads
+    // is written by this call's split kernel first
+    KAP_CUDA(cudaMemsetAsync(base, 0, 256, stream));
+    const int threads = 128;
+    kap_static_build_items_kernel<<<(unsigned)((n_items + threads - 1) / threads), threads, 0, stream>>>(
+        plan_indptr, batch, num_kv_heads, num_splits, reinterpret_cast<WorkItem*>(base + lay.items_off),
+        reinterpret_cast<MergeGroup*>(base + lay.groups_off));
+    KAP_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    // plain launches: the work list was written by the kernel just before, so the split kernel
+    // must not start early
+    kap_attn_split_kernel<<<(unsigned)n_items, kThreads, kSmemBytes, stream>>>(map, p);
+    KAP_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    if (num_splits > 1) {
+        kap_attn_merge_kernel<<<(unsigned)n_groups, 128, 0, stream>>>(p, p.groups);
+        KAP_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+    }
+    if (device_status)
+        KAP_CUDA(cudaMemcpyAsync(device_status, base, sizeof(int32_t), cudaMemcpyDeviceToDevice, stream));
+    return KAP_OK;
+}

@@ -35,6 +35,9 @@ SIGNATURES = {
                                            _vp, _vp, _vp, _vp]),
     "kap_verify_attn": (C.c_int, [_vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_int32, C.c_int32,
                                   C.c_int32, C.c_int32, C.c_int32, C.c_float, _vp, _vp, _vp, _vp]),
+    "kap_selected_decode_attn_static": (C.c_int, [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, C.c_int32,
+                                                  C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                  C.c_float, C.c_int32, _vp, _vp, _vp, _vp]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
     "kap_set_launch_options": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
     "kap_launch_count": (C.c_int64, []),
@@ -218,4 +221,20 @@ def verify_attn(q, q_indptr, kv_pool, bt_indptr, bt_pages, ctx_len, out, ws: Wor
         _dptr(q), _dptr(q_indptr), _dptr(kv_pool), int(pages), _dptr(bt_indptr), _dptr(bt_pages),
         _dptr(ctx_len), int(ctx_len.shape[0]), Hq, Hkv, d, P, sm_scale, _dptr(out), _dptr(lse),
         ws._h, _stream_ptr(stream)))
+    return out
+
+
+def selected_decode_attn_static(q, kv_pool, plan_indptr, plan_phys_pages, plan_logical_pages, ctx_len,
+                                out, num_splits, lse=None, device_status=None, sm_scale=None,
+                                stream=None):
+    """kap_selected_decode_attn_static: the proposal-path attention without a workspace, for
+    callers that may not allocate device memory (scratch is a fixed array inside the library).
+    `device_status`: optional int32 CUDA tensor of one element that receives the status bits."""
+    B, Hq, d = q.shape
+    pages, _, Hkv, P, _ = kv_pool.shape
+    sm_scale = float(d) ** -0.5 if sm_scale is None else float(sm_scale)
+    _check(lib().kap_selected_decode_attn_static(
+        _dptr(q), _dptr(kv_pool), int(pages), _dptr(plan_indptr), _dptr(plan_phys_pages),
+        _dptr(plan_logical_pages), _dptr(ctx_len), B, Hq, Hkv, d, P, sm_scale, int(num_splits),
+        _dptr(out), _dptr(lse), _dptr(device_status), _stream_ptr(stream)))
     return out
