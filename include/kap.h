@@ -86,8 +86,8 @@ enum {
  * Errors: KAP_ERR_INVALID_ARG for batch < 0, page_size <= 0, ctx_len <= 0, a negative budget /
  * sink / recent / span length, a NaN score, a non-monotone span_indptr, a block table shorter than
  * n_pages, a negative block-table entry, or a required pointer that is NULL; KAP_ERR_CAPACITY when
- * the plan needs more than plan_capacity entries (the paper's "plan exceeds the compact workspace"
- * fallback condition).  On any error no output is written.
+ * the plan needs more than plan_capacity entries (one of the paper's fallback conditions: a plan
+ * larger than the space reserved for it).  On any error no output is written.
  */
 kap_status kap_compile_plan(
     int32_t batch, int32_t page_size,
@@ -112,8 +112,8 @@ kap_status kap_compile_plan(
 
 /*
  * Workspace: the split-K work list of one launch shape and the buffers for the partial results
- * (the paper's "reusable workspace" and stable metadata shapes, Section 3.2 "Runtime stability and
- * fallback").  The paper has no counterpart for the split-K schedule itself; it is how this
+ * (Section 3.2 "Runtime stability and fallback" asks for a workspace that is reused and for metadata
+ * whose shapes do not change between steps).  The paper has no counterpart for the split-K schedule itself; it is how this
  * library spreads one sequence's page list over the GPU's SMs.
  *
  * kap_workspace_create allocates (cudaMalloc / cudaMallocHost) on `device`:
