@@ -145,19 +145,23 @@ kap_status kap_schedule(
     int32_t max_chunk_pages,           /* cap on pages per work item, 0 => default */
     void* cuda_stream);
 
-/* The schedule kap_schedule would build for `cta_slots` resident CTAs per wave, written to HOST
+/* The schedule kap_schedule would build for `cta_slots` resident CTAs per wave and clusters of
+ * at most `max_cluster` CTAs (resident clusters approximated as cta_slots / size), written to HOST
  * arrays without touching a GPU (for inspection and tests).  items_out holds max_items rows of
- * 8 int32: seq, kv_head, page_begin, page_end (relative to the sequence's list), group, partial
- * slot, n_splits, n_q; longest chunks first.  Any output pointer may be NULL.  Like kap_schedule
- * it has no counterpart in the paper.  Errors as kap_schedule, minus KAP_ERR_CUDA. */
+ * 8 int32: seq, kv_head, page_begin, page_end (relative to the sequence's list; shared evenly by
+ * the CTAs of the item's cluster), group, partial slot, n_splits, n_q; longest chunks first.
+ * max_chunk = most pages one CTA streams.  Any output pointer may be NULL.  Like kap_schedule it
+ * has no counterpart in the paper.  Errors as kap_schedule, minus KAP_ERR_CUDA. */
 kap_status kap_schedule_host(
     int32_t batch, const int32_t* list_len, const int32_t* n_q, int32_t num_q_heads,
-    int32_t num_kv_heads, int32_t cta_slots, int32_t max_chunk_pages, int32_t max_items,
-    int32_t* items_out, int32_t* n_items, int32_t* n_merge_groups, int32_t* max_chunk);
+    int32_t num_kv_heads, int32_t cta_slots, int32_t max_cluster, int32_t max_chunk_pages,
+    int32_t max_items, int32_t* items_out, int32_t* n_items, int32_t* n_merge_groups,
+    int32_t* max_chunk, int32_t* cluster_size);
 
 /* what the last kap_schedule produced; any pointer may be NULL */
 kap_status kap_schedule_info(const kap_workspace* ws, int32_t* n_items, int32_t* n_merge_groups,
-                             int32_t* max_chunk_pages, int32_t* ctas_per_wave);
+                             int32_t* max_chunk_pages, int32_t* ctas_per_wave,
+                             int32_t* cluster_size);
 
 /*
  * kap_selected_decode_attn - Section 3.2 "Selected-KV proposal".  For sequence b and query head h
@@ -165,7 +169,8 @@ kap_status kap_schedule_info(const kap_workspace* ws, int32_t* n_items, int32_t*
  *     z_t = sm_scale * <q[b,h,:], K[g,t,:]>,   out[b,h,:] = sum_t softmax_t(z) V[g,t,:],
  *     lse[b,h] = ln sum_t exp(z_t)            (natural log)
  * computed as split-K flash decoding (bf16 tensor-core products, fp32 accumulation, base-2 online
- * softmax) followed by a log-sum-exp merge of the splits.  One layer per call.
+ * softmax); the splits' results are merged by log-sum-exp, inside a thread-block cluster through
+ * distributed shared memory and, for lists too long for one cluster, by a separate merge pass.  One layer per call.
  * plan_logical_pages == NULL means "logical page = position in the list" (identity plan).
  * The plan arrays are the DEVICE copies of kap_compile_plan's outputs; `ws` must hold a schedule
  * made from the same per-sequence list lengths with n_q = NULL.
@@ -278,13 +283,15 @@ kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);
  *                (t < ctx_len - n_q) - pages written in earlier decoding steps.  ctx_len and those
  *                pages must then be final before the previous kernel was launched; Q, the pages
  *                holding the rows' own tokens, out and lse may still be written by it.
- *   fused_merge  != 0: the last split of a (sequence, KV head) to finish merges the splits inside
- *                the split kernel instead of launching the separate merge pass (default 0).
  *   ctas_per_sm  resident CTAs per SM the scheduler fills in one wave; 0 = as many as fit.
- *                Takes effect at the next kap_schedule.
- * The paper has no counterpart for these. */
-kap_status kap_set_launch_options(int32_t use_pdl, int32_t fused_merge, int32_t ctas_per_sm,
-                                  int32_t early_kv);
+ *   max_cluster  largest thread-block cluster (1, 2, 4 or 8; default 8) the scheduler may give a
+ *                work item.  The CTAs of a cluster share the item's pages and reduce their partial
+ *                results through distributed shared memory, so a (sequence, KV head) that fits one
+ *                cluster needs no merge pass.
+ * ctas_per_sm and max_cluster take effect at the next kap_schedule.  The paper has no counterpart
+ * for these.  Error: KAP_ERR_INVALID_ARG for a max_cluster that is not 1, 2, 4 or 8. */
+kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, int32_t ctas_per_sm,
+                                  int32_t max_cluster);
 
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t kap_launch_count(void);

@@ -32,10 +32,10 @@
 namespace kap {
 
 kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t* n_q,
-                          int32_t num_q_heads, int32_t num_kv_heads, int32_t cta_slots,
+                          int32_t num_q_heads, int32_t num_kv_heads, const int32_t cluster_slots[4],
                           int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
                           std::vector<WorkItem>& items, std::vector<MergeGroup>& groups,
-                          int32_t* max_chunk_out, int32_t* row_tiles_out);
+                          int32_t* max_chunk_out, int32_t* row_tiles_out, int32_t* cluster_out);
 
 // ------------------------------------------------------------------------------ kernel geometry
 constexpr int kWarps = 4;
@@ -56,7 +56,8 @@ struct SmemTail {                                         // what follows the ri
     unsigned long long empty[kSlots];
     float m[kWarps][kRowTile];
     float l[kWarps][kRowTile];
-    int32_t is_last;
+    float cta_m[kRowTile * kMaxRowTiles];     // CTA-level state read by cluster peers
+    float cta_l[kRowTile * kMaxRowTiles];
     int32_t timed_out;
 };
 constexpr int kSmemBytes = kRingBytes + (int)sizeof(SmemTail) + 1024;   // + alignment slack
@@ -75,13 +76,12 @@ struct AttnParams {
     const MergeGroup* groups;
     float* part_o;                   // [slots][rows_cap][128]
     float* part_ml;                  // [slots][rows_cap][2]
-    int32_t* counters;               // [groups] arrival counters (fused merge)
     __nv_bfloat16* out;              // [rows, Hq, d]
     float* lse;                      // [rows, Hq] or null
     int32_t* status;
     long long num_pool_pages;
     int32_t Hq, Hkv, G, rows_cap;
-    int32_t fused_merge, early_kv;
+    int32_t cluster, early_kv;       // CTAs per work item (cluster size); early KV prefetch
     float scale_log2;                // sm_scale * log2(e)
 #ifdef KAP_TRACE
     unsigned long long* trace;       // [8192 records][8] timestamps of this launch (debug builds)
@@ -171,6 +171,27 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+// Thread-block clusters: barrier over all threads of all CTAs of the cluster (release / acquire),
+// and loads from a peer CTA's shared memory (distributed shared memory).
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta_rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
+    return r;
+}
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_dsmem_f32x4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
 // Programmatic dependent launch: let the next kernel on the stream start its prologue now ...
 __device__ __forceinline__ void pdl_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -205,33 +226,28 @@ __device__ __forceinline__ void store_final(const AttnParams& p, int64_t q_row, 
         p.lse[q_row * p.Hq + head] = r.l > 0.f ? (r.m + log2f(r.l)) * 0.6931471805599453f : -INFINITY;
 }
 
-// Merge the splits of one group and write its final rows.  `tid` / `nthreads` enumerate the
-// calling threads; each handles (row, 4-column) cells.  The partials are read in batches of
-// independent loads so that a cell costs one memory round trip per batch.
-__device__ __forceinline__ void merge_group_splits(const AttnParams& p, const MergeGroup& g,
-                                                   int64_t q_row0, int tid, int nthreads) {
+// Merge the splits of one group for one (row, 4-column) cell and write the final values.  The
+// partials are read in batches of independent loads: one memory round trip per batch.
+__device__ __forceinline__ void merge_group_cell(const AttnParams& p, const MergeGroup& g,
+                                                 int64_t q_row0, int R, int c4) {
     constexpr int kBatch = 8;
-    const int rows = g.n_q * p.G;
-    for (int idx = tid; idx < rows * 32; idx += nthreads) {
-        const int R = idx >> 5, c4 = idx & 31;
-        const int64_t base = (int64_t)g.first_item * p.rows_cap + R;
-        const int64_t stride = p.rows_cap;
-        Merged r; r.m = -INFINITY; r.l = 0.f; r.o = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int i0 = 0; i0 < g.n_splits; i0 += kBatch) {
-            float2 ml[kBatch];
-            float4 o[kBatch];
+    const int64_t base = (int64_t)g.first_item * p.rows_cap + R;
+    const int64_t stride = p.rows_cap;
+    Merged r; r.m = -INFINITY; r.l = 0.f; r.o = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i0 = 0; i0 < g.n_splits; i0 += kBatch) {
+        float2 ml[kBatch];
+        float4 o[kBatch];
 #pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                const int i = min(i0 + j, g.n_splits - 1);
-                ml[j] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + i * stride) * 2));
-                o[j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (base + i * stride) * kHeadDim) + c4);
-            }
-#pragma unroll
-            for (int j = 0; j < kBatch; ++j)
-                if (i0 + j < g.n_splits) merge_into(r, ml[j].x, ml[j].y, o[j]);
+        for (int j = 0; j < kBatch; ++j) {
+            const int i = min(i0 + j, g.n_splits - 1);
+            ml[j] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + i * stride) * 2));
+            o[j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (base + i * stride) * kHeadDim) + c4);
         }
-        store_final(p, q_row0 + R / p.G, g.kv_head * p.G + R % p.G, c4, r);
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j)
+            if (i0 + j < g.n_splits) merge_into(r, ml[j].x, ml[j].y, o[j]);
     }
+    store_final(p, q_row0 + R / p.G, g.kv_head * p.G + R % p.G, c4, r);
 }
 
 // ------------------------------------------------------------------------------ the split kernel
@@ -254,7 +270,15 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
 
     // ---- prologue on static metadata only (work list, page lists, q_indptr): with programmatic
     // dependent launch it overlaps the tail of the previous kernel on the stream.
-    const WorkItem item = p.items[blockIdx.x];
+    // A work item belongs to a cluster of C CTAs (C = 1: no cluster); CTA `rank` takes its even
+    // share of the item's pages.
+    const int C = p.cluster, rank = blockIdx.x % C;
+    WorkItem item = p.items[blockIdx.x / C];
+    {
+        const int n = item.page_end - item.page_begin, base = n / C, rem = n % C;
+        item.page_begin += rank * base + min(rank, rem);
+        item.page_end = item.page_begin + base + (rank < rem ? 1 : 0);
+    }
     const int n_pages = item.page_end - item.page_begin;
     const int rows = item.n_q * p.G;                         // valid query rows of this item
     int RT = (rows + kRowTile - 1) / kRowTile;               // row tiles: 1, 2 or 4
@@ -264,7 +288,6 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             mbar_init(smem_u32(&tail->full[s]), 1);
             mbar_init(smem_u32(&tail->empty[s]), RT);
         }
-        tail->is_last = 0;
         tail->timed_out = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map) : "memory");
@@ -480,8 +503,13 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     }
     __syncthreads();
 
-    const float* all = reinterpret_cast<const float*>(ring);
+    float* all = reinterpret_cast<float*>(ring);
+    float* m_flat = tail->cta_m;
+    float* l_flat = tail->cta_l;
     const bool single = item.n_splits == 1;
+    // Combine the warp groups: the CTA-level state of row R ends up in scratch row R (the region
+    // of warp R / 16 of group 0, which only this cell's thread reads) and cta_m[R], cta_l[R]; with
+    // one CTA per item it goes straight to global memory instead.
     for (int idx = tid; idx < rows * 32; idx += kThreads) {
         const int R = idx >> 5, c4 = idx & 31;
         const int t = R / kRowTile, r = R % kRowTile;
@@ -491,13 +519,45 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             merge_into(res, tail->m[w][r], tail->l[w][r],
                        *reinterpret_cast<const float4*>(all + (w * kRowTile + r) * kScratchStride + c4 * 4));
         }
-        if (single) {
-            store_final(p, q_row0 + R / p.G, item.kv_head * p.G + R % p.G, c4, res);
+        if (C == 1) {
+            if (single) {
+                store_final(p, q_row0 + R / p.G, item.kv_head * p.G + R % p.G, c4, res);
+            } else {
+                const int64_t prow = (int64_t)item.split * p.rows_cap + R;
+                *(reinterpret_cast<float4*>(p.part_o + prow * kHeadDim) + c4) = res.o;
+                if (c4 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(res.m, res.l);
+            }
         } else {
-            const int64_t prow = (int64_t)item.split * p.rows_cap + R;
-            *(reinterpret_cast<float4*>(p.part_o + prow * kHeadDim) + c4) = res.o;
-            if (c4 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(res.m, res.l);
+            *reinterpret_cast<float4*>(all + R * kScratchStride + c4 * 4) = res.o;
+            if (c4 == 0) { m_flat[R] = res.m; l_flat[R] = res.l; }
         }
+    }
+    if (C > 1) {
+        // Cluster reduction through distributed shared memory: after the first cluster barrier
+        // every CTA's state is visible to its peers; rank r merges its share of the (row, column)
+        // cells over all C CTAs and writes them out; the second barrier keeps every CTA's shared
+        // memory alive until all peers have read it.
+        cluster_sync();
+        const int n_cells = rows * 32;
+        const int per_rank = (n_cells + C - 1) / C;
+        const int c_end = min(n_cells, (rank + 1) * per_rank);
+        for (int idx = rank * per_rank + tid; idx < c_end; idx += kThreads) {
+            const int R = idx >> 5, c4 = idx & 31;
+            Merged res; res.m = -INFINITY; res.l = 0.f; res.o = make_float4(0.f, 0.f, 0.f, 0.f);
+            const uint32_t o_addr = smem_u32(all + R * kScratchStride + c4 * 4);
+            const uint32_t m_addr = smem_u32(m_flat + R), l_addr = smem_u32(l_flat + R);
+            for (int peer = 0; peer < C; ++peer)
+                merge_into(res, ld_dsmem_f32(map_to_cta(m_addr, peer)), ld_dsmem_f32(map_to_cta(l_addr, peer)),
+                           ld_dsmem_f32x4(map_to_cta(o_addr, peer)));
+            if (single) {
+                store_final(p, q_row0 + R / p.G, item.kv_head * p.G + R % p.G, c4, res);
+            } else {
+                const int64_t prow = (int64_t)item.split * p.rows_cap + R;
+                *(reinterpret_cast<float4*>(p.part_o + prow * kHeadDim) + c4) = res.o;
+                if (c4 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(res.m, res.l);
+            }
+        }
+        cluster_sync();
     }
     KAP_TRACE_POINT(blockIdx.x, 5);
 #ifdef KAP_TRACE
@@ -507,26 +567,11 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         p.trace[(size_t)blockIdx.x * 8 + 7] = smid;
     }
 #endif
-    if (single || !p.fused_merge) return;
-
-    // Fused merge: the last split of the group to arrive combines all of them.
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int prev = atomicAdd(p.counters + item.group, 1);
-        const int last = prev == item.n_splits - 1;
-        if (last) p.counters[item.group] = 0;           // leave the counter clean for the next launch
-        tail->is_last = last;
-    }
-    __syncthreads();
-    if (!tail->is_last) return;
-    __threadfence();
-    merge_group_splits(p, p.groups[item.group], q_row0, tid, kThreads);
-    KAP_TRACE_POINT(blockIdx.x, 6);
 }
 
 // -------------------------------------------------------------------- the separate merge kernel
-// One CTA per (sequence, KV head) that has more than one split.
+// grid.x = (sequence, KV head) groups that have more than one split, grid.y = blocks of 4 query
+// rows; 128 threads = 4 rows x 32 four-column cells, one cell per thread.
 __global__ void __launch_bounds__(128)
 kap_attn_merge_kernel(const AttnParams p, const MergeGroup* merge_groups)
 {
@@ -534,9 +579,10 @@ kap_attn_merge_kernel(const AttnParams p, const MergeGroup* merge_groups)
     KAP_TRACE_POINT(4096 + blockIdx.x, 0);
     const MergeGroup g = merge_groups[blockIdx.x];          // static metadata: before the wait
     const int64_t q_row0 = p.q_indptr ? p.q_indptr[g.seq] : g.seq;
+    const int R = blockIdx.y * 4 + (threadIdx.x >> 5), c4 = threadIdx.x & 31;
     pdl_wait();
     KAP_TRACE_POINT(4096 + blockIdx.x, 2);
-    merge_group_splits(p, g, q_row0, threadIdx.x, blockDim.x);
+    if (R < g.n_q * p.G) merge_group_cell(p, g, q_row0, R, c4);
     KAP_TRACE_POINT(4096 + blockIdx.x, 5);
 }
 
@@ -545,7 +591,7 @@ namespace {
 
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_use_pdl{1};
-std::atomic<int> g_fused_merge{0};
+std::atomic<int> g_max_cluster{8};       // largest thread-block cluster the scheduler may pick
 std::atomic<int> g_early_kv{1};
 std::atomic<int> g_ctas_per_sm{0};       // 0 = as many as fit (occupancy)
 
@@ -627,27 +673,41 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
         return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(g_attr_err));
 
     AttnParams p = p_in;
-    p.fused_merge = g_fused_merge.load() ? 1 : 0;
+    p.cluster = ws->cluster_size;
     p.early_kv = (g_use_pdl.load() && g_early_kv.load()) ? 1 : 0;
 #ifdef KAP_TRACE
     p.trace = (g_trace && g_trace_next < g_trace_cap) ? g_trace + (size_t)(g_trace_next++) * 8192 * 8 : nullptr;
 #endif
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (g_use_pdl.load()) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    const int n_pdl_attr = n_attr;
+    if (ws->cluster_size > 1) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = (unsigned)ws->cluster_size;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)ws->n_items);
+    cfg.gridDim = dim3((unsigned)ws->n_items * (unsigned)ws->cluster_size);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
     cfg.attrs = attr;
-    cfg.numAttrs = g_use_pdl.load() ? 1 : 0;
+    cfg.numAttrs = n_attr;
     KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel, *map, p));
     g_launches.fetch_add(1);
-    if (!p.fused_merge && ws->n_merge_groups > 0) {
-        cfg.gridDim = dim3((unsigned)ws->n_merge_groups);
+    if (ws->n_merge_groups > 0) {
+        const int rows = ws->max_nq * p.G;
+        cfg.gridDim = dim3((unsigned)ws->n_merge_groups, (unsigned)((rows + 3) / 4));
         cfg.blockDim = dim3(128);
         cfg.dynamicSmemBytes = 0;
+        cfg.numAttrs = n_pdl_attr;
         const MergeGroup* mg = ws->d_merge;
         KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_merge_kernel, p, mg));
         g_launches.fetch_add(1);
@@ -703,13 +763,11 @@ extern "C" kap_status kap_workspace_create(kap_workspace** out, int32_t device, 
     dev((void**)&ws->d_merge, sizeof(MergeGroup) * max_groups);
     dev((void**)&ws->d_part_o, sizeof(float) * (size_t)max_items * max_rows_per_item * kHeadDim);
     dev((void**)&ws->d_part_ml, sizeof(float) * (size_t)max_items * max_rows_per_item * 2);
-    dev((void**)&ws->d_counters, sizeof(int32_t) * max_groups);
     dev((void**)&ws->d_status, sizeof(int32_t));
     host((void**)&ws->h_items, sizeof(WorkItem) * max_items);
     host((void**)&ws->h_groups, sizeof(MergeGroup) * max_groups);
     host((void**)&ws->h_merge, sizeof(MergeGroup) * max_groups);
     host((void**)&ws->h_status, sizeof(int32_t));
-    if (e == cudaSuccess) e = cudaMemset(ws->d_counters, 0, sizeof(int32_t) * max_groups);
     if (e == cudaSuccess) e = cudaMemset(ws->d_status, 0, sizeof(int32_t));
     cudaEvent_t ev = nullptr;
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
@@ -727,6 +785,21 @@ extern "C" kap_status kap_workspace_create(kap_workspace** out, int32_t device, 
         per_sm = 1;
     ws->occupancy = per_sm;
     ws->ctas_per_wave = per_sm * ws->sm_count;
+    // how many clusters of 2, 4, 8 CTAs can be resident at once (GPC boundaries cost a few)
+    for (int ci = 1; ci < 4; ++ci) {
+        cudaLaunchAttribute ca[1];
+        ca[0].id = cudaLaunchAttributeClusterDimension;
+        ca[0].val.clusterDim.x = 1u << ci; ca[0].val.clusterDim.y = 1; ca[0].val.clusterDim.z = 1;
+        cudaLaunchConfig_t cc{};
+        cc.gridDim = dim3((unsigned)(ws->sm_count * per_sm / (1 << ci)) * (1u << ci));
+        cc.blockDim = dim3(kThreads);
+        cc.dynamicSmemBytes = kSmemBytes;
+        cc.attrs = ca; cc.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
+        ws->max_clusters[ci] = n;
+    }
+    ws->max_clusters[0] = ws->ctas_per_wave;
     *out = ws;
     return KAP_OK;
 }
@@ -734,7 +807,7 @@ extern "C" kap_status kap_workspace_create(kap_workspace** out, int32_t device, 
 extern "C" void kap_workspace_destroy(kap_workspace* ws) {
     if (!ws) return;
     cudaFree(ws->d_items); cudaFree(ws->d_groups); cudaFree(ws->d_merge); cudaFree(ws->d_part_o);
-    cudaFree(ws->d_part_ml); cudaFree(ws->d_counters); cudaFree(ws->d_status);
+    cudaFree(ws->d_part_ml); cudaFree(ws->d_status);
     cudaFreeHost(ws->h_items); cudaFreeHost(ws->h_groups); cudaFreeHost(ws->h_merge);
     cudaFreeHost(ws->h_status);
     if (ws->upload_event) cudaEventDestroy((cudaEvent_t)ws->upload_event);
@@ -750,11 +823,21 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     std::vector<WorkItem> items;
     std::vector<MergeGroup> groups;
     int32_t max_chunk = 0, row_tiles = 1;
+    // resident slots per cluster size: all of the SM's CTA slots, or ctas_per_sm of them
     const int want = g_ctas_per_sm.load();
-    ws->ctas_per_wave = (want > 0 ? std::min(want, ws->occupancy) : ws->occupancy) * ws->sm_count;
-    kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, ws->ctas_per_wave,
+    const int per_sm = want > 0 ? std::min(want, ws->occupancy) : ws->occupancy;
+    ws->ctas_per_wave = per_sm * ws->sm_count;
+    int32_t slots[4];
+    for (int ci = 0; ci < 4; ++ci) {
+        const int c = 1 << ci;
+        const int64_t scaled = (int64_t)ws->max_clusters[ci] * per_sm / ws->occupancy;
+        slots[ci] = c <= g_max_cluster.load() ? (int32_t)std::min<int64_t>(scaled, ws->ctas_per_wave / c) : 0;
+    }
+    slots[0] = ws->ctas_per_wave;
+    int32_t cluster = 1;
+    kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots,
                                    max_chunk_pages, ws->max_items, ws->max_rows, items, groups,
-                                   &max_chunk, &row_tiles);
+                                   &max_chunk, &row_tiles, &cluster);
     if (st != KAP_OK) return st;
     if ((int64_t)items.size() > ws->max_items || (int64_t)groups.size() > ws->max_items)
         return fail(KAP_ERR_CAPACITY, "%zu work items exceed the workspace's %d", items.size(), ws->max_items);
@@ -783,18 +866,22 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     ws->batch = batch; ws->n_items = (int32_t)items.size(); ws->n_groups = (int32_t)groups.size();
     ws->n_merge_groups = n_merge; ws->max_chunk = max_chunk; ws->row_tiles = row_tiles;
     ws->num_q_heads = num_q_heads; ws->num_kv_heads = num_kv_heads; ws->has_nq = n_q != nullptr;
-    ws->total_rows = total_rows;
+    ws->total_rows = total_rows; ws->cluster_size = cluster;
+    int32_t mq = 1;
+    for (int32_t b = 0; b < batch; ++b) mq = std::max(mq, n_q ? n_q[b] : 1);
+    ws->max_nq = mq;
     return KAP_OK;
 }
 
 extern "C" kap_status kap_schedule_info(const kap_workspace* ws, int32_t* n_items,
                                         int32_t* n_merge_groups, int32_t* max_chunk_pages,
-                                        int32_t* ctas_per_wave) {
+                                        int32_t* ctas_per_wave, int32_t* cluster_size) {
     if (!ws) return fail(KAP_ERR_INVALID_ARG, "NULL workspace");
     if (n_items) *n_items = ws->n_items;
     if (n_merge_groups) *n_merge_groups = ws->n_merge_groups;
     if (max_chunk_pages) *max_chunk_pages = ws->max_chunk;
     if (ctas_per_wave) *ctas_per_wave = ws->ctas_per_wave;
+    if (cluster_size) *cluster_size = ws->cluster_size;
     return KAP_OK;
 }
 
@@ -802,7 +889,7 @@ static AttnParams base_params(kap_workspace* ws, int32_t hq, int32_t hkv, float 
                               int64_t num_pool_pages) {
     AttnParams p{};
     p.items = ws->d_items; p.groups = ws->d_groups; p.part_o = ws->d_part_o;
-    p.part_ml = ws->d_part_ml; p.counters = ws->d_counters; p.status = ws->d_status;
+    p.part_ml = ws->d_part_ml; p.status = ws->d_status;
     p.num_pool_pages = num_pool_pages; p.Hq = hq; p.Hkv = hkv; p.G = hq / hkv;
     p.rows_cap = ws->max_rows;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
@@ -857,12 +944,14 @@ extern "C" kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream) 
     return KAP_OK;
 }
 
-extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t fused_merge, int32_t ctas_per_sm,
-                                             int32_t early_kv) {
-    if (early_kv >= 0) g_early_kv.store(early_kv ? 1 : 0);
+extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, int32_t ctas_per_sm,
+                                             int32_t max_cluster) {
+    if (max_cluster == 0 || max_cluster > 8 || (max_cluster > 0 && (max_cluster & (max_cluster - 1))))
+        return fail(KAP_ERR_INVALID_ARG, "max_cluster %d (allowed: 1, 2, 4, 8)", max_cluster);
     if (use_pdl >= 0) g_use_pdl.store(use_pdl ? 1 : 0);
-    if (fused_merge >= 0) g_fused_merge.store(fused_merge ? 1 : 0);
+    if (early_kv >= 0) g_early_kv.store(early_kv ? 1 : 0);
     if (ctas_per_sm >= 0) g_ctas_per_sm.store(ctas_per_sm);
+    if (max_cluster > 0) g_max_cluster.store(max_cluster);
     return KAP_OK;
 }
 
@@ -1012,11 +1101,10 @@ extern "C" kap_status kap_selected_decode_attn_static(
     p.groups = reinterpret_cast<const MergeGroup*>(base + lay.groups_off);
     p.part_ml = reinterpret_cast<float*>(base + lay.ml_off);
     p.part_o = reinterpret_cast<float*>(base + lay.o_off);
-    p.counters = nullptr;
     p.out = (__nv_bfloat16*)out; p.lse = lse;
     p.status = reinterpret_cast<int32_t*>(base);
     p.num_pool_pages = num_pool_pages; p.Hq = num_q_heads; p.Hkv = num_kv_heads; p.G = rows;
-    p.rows_cap = rows; p.fused_merge = 0; p.early_kv = 0;
+    p.rows_cap = rows; p.cluster = 1; p.early_kv = 0;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
 #ifdef KAP_TRACE
     p.trace = nullptr;
@@ -1038,7 +1126,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
     KAP_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     if (num_splits > 1) {
-        kap_attn_merge_kernel<<<(unsigned)n_groups, 128, 0, stream>>>(p, p.groups);
+        kap_attn_merge_kernel<<<dim3((unsigned)n_groups, (unsigned)((rows + 3) / 4)), 128, 0, stream>>>(p, p.groups);
         KAP_CUDA(cudaGetLastError());
         g_launches.fetch_add(1);
     }

@@ -44,6 +44,8 @@ struct kap_workspace {
     int32_t device = 0;
     int32_t max_items = 0, max_rows = 0, max_batch = 0;
     int32_t sm_count = 0, occupancy = 1;
+    int32_t max_clusters[4] = {0, 0, 0, 0};  // resident clusters of 1, 2, 4, 8 CTAs
+    int32_t cluster_size = 1, max_nq = 1;    // of the last schedule
     // last schedule
     int32_t batch = 0, n_items = 0, n_groups = 0, n_merge_groups = 0, max_chunk = 0;
     int32_t ctas_per_wave = 0, row_tiles = 1, num_q_heads = 0, num_kv_heads = 0;
@@ -60,7 +62,6 @@ struct kap_workspace {
     int32_t* d_qrow0 = nullptr;
     float* d_part_o = nullptr;               // [max_items][max_rows][128]
     float* d_part_ml = nullptr;              // [max_items][max_rows][2]   (m in log2 units, l)
-    int32_t* d_counters = nullptr;           // [max groups] arrival counters (fused merge)
     int32_t* d_status = nullptr;             // device status word
     int32_t* h_status = nullptr;             // pinned read-back
     void* upload_event = nullptr;            // cudaEvent_t: last schedule upload done

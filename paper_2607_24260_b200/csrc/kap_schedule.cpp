@@ -3,8 +3,9 @@
 // The paper (Section 3.2, "Runtime stability and fallback") asks for stable metadata shapes so
 // that decode steps replay as CUDA graphs; it does not describe how one sequence's pages are
 // spread over a GPU.  This file is that part: every (sequence, KV head) page list is cut into
-// near-equal contiguous chunks, one chunk per CTA, such that the chunks fill the GPU's resident
-// CTA slots in whole waves.  The result depends only on page counts and row counts, so it is
+// near-equal contiguous chunks, one chunk per thread-block cluster (whose CTAs share it evenly and
+// reduce their partial results through distributed shared memory), such that the clusters fill
+// the GPU's resident slots in whole waves.  The result depends only on page counts and row counts, so it is
 // computed once per request shape and reused for every layer and step.
 #include <algorithm>
 #include <cstring>
@@ -26,24 +27,28 @@ int64_t chunks_for(const int32_t* len, int32_t batch, int32_t hkv, int64_t t) {
 
 }  // namespace
 
-// Cost model used to pick the number of waves: a CTA pays a fixed start-up/epilogue cost worth
-// about kFixedPages pages of streaming, waves run back to back.
+// Cost model used to pick the cluster size and the number of waves, in units of "pages streamed
+// by one CTA": a CTA pays a fixed start-up / epilogue cost, a launch whose groups need more than
+// one cluster pays for the separate merge pass, a cluster pays for its two cluster barriers.
 constexpr int64_t kFixedPages = 6;
-constexpr int32_t kDefaultChunkCap = 512;     // also the size of the kernel's page-id buffer
+constexpr int64_t kMergePassPages = 9;
+constexpr int64_t kClusterPages = 1;
+constexpr int32_t kDefaultChunkCap = 512;     // per CTA; also the size of the kernel's page-id buffer
 
+// cluster_slots[i] = clusters of size 1 << i that can be resident at once (0 = size not allowed)
 kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t* n_q,
-                          int32_t num_q_heads, int32_t num_kv_heads, int32_t cta_slots,
+                          int32_t num_q_heads, int32_t num_kv_heads, const int32_t cluster_slots[4],
                           int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
                           std::vector<WorkItem>& items, std::vector<MergeGroup>& groups,
-                          int32_t* max_chunk_out, int32_t* row_tiles_out)
+                          int32_t* max_chunk_out, int32_t* row_tiles_out, int32_t* cluster_out)
 {
     if (batch < 0 || (batch > 0 && !list_len)) return fail(KAP_ERR_INVALID_ARG, "bad batch / list_len");
     if (num_q_heads <= 0 || num_kv_heads <= 0 || num_q_heads % num_kv_heads)
         return fail(KAP_ERR_INVALID_ARG, "head counts %d / %d", num_q_heads, num_kv_heads);
     const int32_t G = num_q_heads / num_kv_heads;
     if (kRowTile % G) return fail(KAP_ERR_UNSUPPORTED, "group size %d must divide %d", G, kRowTile);
-    if (cta_slots <= 0) return fail(KAP_ERR_INVALID_ARG, "cta_slots %d", cta_slots);
-    int32_t cap = max_chunk_pages <= 0 ? kDefaultChunkCap : std::min(max_chunk_pages, kDefaultChunkCap);
+    if (cluster_slots[0] <= 0) return fail(KAP_ERR_INVALID_ARG, "cta_slots %d", cluster_slots[0]);
+    const int32_t cap = max_chunk_pages <= 0 ? kDefaultChunkCap : std::min(max_chunk_pages, kDefaultChunkCap);
     int32_t max_len = 0, max_nq = 1;
     for (int32_t b = 0; b < batch; ++b) {
         if (list_len[b] <= 0) return fail(KAP_ERR_INVALID_ARG, "list_len[%d] = %d <= 0", b, list_len[b]);
@@ -62,9 +67,10 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
     groups.clear();
     *max_chunk_out = 0;
     *row_tiles_out = row_tiles;
+    *cluster_out = 1;
     if (batch == 0) return KAP_OK;
 
-    // smallest chunk size t with chunks_for(t) <= slots * waves, for the cheapest wave count
+    // smallest cluster-level chunk t with chunks_for(t) <= budget clusters
     auto min_chunk = [&](int64_t budget) -> int64_t {
         int64_t lo = 1, hi = max_len;
         if (chunks_for(list_len, batch, num_kv_heads, hi) > budget) return -1;
@@ -75,23 +81,34 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
         return lo;
     };
     int64_t best_t = -1, best_cost = INT64_MAX;
+    int32_t best_c = 1;
     const int64_t item_cap = std::max<int64_t>(1, max_items);
-    for (int64_t waves = 1; waves <= 64; ++waves) {
-        const int64_t budget = std::min<int64_t>(item_cap, (int64_t)cta_slots * waves);
-        const int64_t t = min_chunk(budget);
-        if (t > 0 && t <= cap) {
-            const int64_t cost = waves * (t + kFixedPages);
-            if (cost < best_cost) { best_cost = cost; best_t = t; }
-            if (t == 1) break;
+    for (int ci = 0; ci < 4; ++ci) {
+        const int64_t C = 1 << ci;
+        if (cluster_slots[ci] <= 0) continue;
+        auto consider = [&](int64_t t, int64_t waves) {
+            if (t <= 0 || (t + C - 1) / C > cap) return false;
+            const bool merge_pass = t < max_len;            // some group needs more than one cluster
+            const int64_t cost = waves * ((t + C - 1) / C + kFixedPages) + (merge_pass ? kMergePassPages : 0)
+                                 + (C > 1 ? kClusterPages : 0);
+            if (cost < best_cost) { best_cost = cost; best_t = t; best_c = (int32_t)C; }
+            return true;
+        };
+        bool found = false;
+        for (int64_t waves = 1; waves <= 64; ++waves) {
+            const int64_t budget = std::min<int64_t>(item_cap, (int64_t)cluster_slots[ci] * waves);
+            const int64_t t = min_chunk(budget);
+            if (consider(t, waves)) { found = true; if (t <= C) break; }
+            if (budget == item_cap) break;                   // no further items to hand out
         }
-        if (budget == item_cap) break;                 // no further items to hand out
-    }
-    if (best_t < 0) {                                   // very long lists: as many items as allowed
-        const int64_t t = min_chunk(item_cap);
-        if (t > 0 && t <= cap) best_t = t;
+        if (!found) consider(min_chunk(item_cap), (item_cap + cluster_slots[ci] - 1) / cluster_slots[ci]);
+        // one cluster per (sequence, KV head): slightly longer chunks, but no merge pass
+        const int64_t n_groups = (int64_t)batch * num_kv_heads;
+        if (n_groups <= item_cap)
+            consider(max_len, (n_groups + cluster_slots[ci] - 1) / cluster_slots[ci]);
     }
     if (best_t < 0)
-        return fail(KAP_ERR_CAPACITY, "page lists need more than %d work items of <= %d pages",
+        return fail(KAP_ERR_CAPACITY, "page lists need more than %d work items of <= %d pages per CTA",
                     max_items, cap);
 
     int32_t slot = 0;
@@ -112,12 +129,13 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
                 it.seq = b; it.kv_head = g; it.page_begin = begin; it.page_end = begin + n;
                 it.group = group_index; it.split = slot; it.n_splits = n_splits; it.n_q = mg.n_q;
                 items.push_back(it);
-                *max_chunk_out = std::max(*max_chunk_out, n);
+                *max_chunk_out = std::max(*max_chunk_out, (n + best_c - 1) / best_c);
                 begin += n;
                 ++slot;
             }
         }
     }
+    *cluster_out = best_c;
     // longest chunks first: the hardware hands out CTAs in index order, so the tail of the last
     // wave is made of the shortest chunks.  WorkItem::split holds the item's partial-result slot
     // (group.first_item + split index), which is what keeps a group's partials contiguous.
@@ -130,19 +148,21 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
 }  // namespace kap
 
 // Exposed for tests and tools: the same schedule kap_schedule uploads, written to HOST arrays.
-// items_out holds max_items rows of 8 int32 (seq, kv_head, page_begin, page_end, group, slot,
-// n_splits, n_q).  Not a paper operation (see the file header).
+// Not a paper operation (see the file header).
 extern "C" kap_status kap_schedule_host(
     int32_t batch, const int32_t* list_len, const int32_t* n_q, int32_t num_q_heads,
-    int32_t num_kv_heads, int32_t cta_slots, int32_t max_chunk_pages, int32_t max_items,
-    int32_t* items_out, int32_t* n_items, int32_t* n_merge_groups, int32_t* max_chunk)
+    int32_t num_kv_heads, int32_t cta_slots, int32_t max_cluster, int32_t max_chunk_pages,
+    int32_t max_items, int32_t* items_out, int32_t* n_items, int32_t* n_merge_groups,
+    int32_t* max_chunk, int32_t* cluster_size)
 {
     std::vector<kap::WorkItem> items;
     std::vector<kap::MergeGroup> groups;
-    int32_t mc = 0, rt = 1;
-    kap_status st = kap::build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, cta_slots,
+    int32_t mc = 0, rt = 1, cl = 1;
+    int32_t slots[4];
+    for (int i = 0; i < 4; ++i) slots[i] = (1 << i) <= std::max(max_cluster, 1) ? cta_slots / (1 << i) : 0;
+    kap_status st = kap::build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots,
                                         max_chunk_pages, max_items, kap::kRowTile * kap::kMaxRowTiles,
-                                        items, groups, &mc, &rt);
+                                        items, groups, &mc, &rt, &cl);
     if (st != KAP_OK) return st;
     if ((int64_t)items.size() > max_items)
         return kap::fail(KAP_ERR_CAPACITY, "%zu items > max_items %d", items.size(), max_items);
@@ -155,5 +175,6 @@ extern "C" kap_status kap_schedule_host(
         *n_merge_groups = n;
     }
     if (max_chunk) *max_chunk = mc;
+    if (cluster_size) *cluster_size = cl;
     return KAP_OK;
 }

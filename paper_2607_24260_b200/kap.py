@@ -28,8 +28,9 @@ SIGNATURES = {
     "kap_workspace_destroy": (None, [_vp]),
     "kap_schedule": (C.c_int, [_vp, C.c_int32, _i32p, _i32p, C.c_int32, C.c_int32, C.c_int32, _vp]),
     "kap_schedule_host": (C.c_int, [C.c_int32, _i32p, _i32p, C.c_int32, C.c_int32, C.c_int32,
-                                    C.c_int32, C.c_int32, _i32p, _i32p, _i32p, _i32p]),
-    "kap_schedule_info": (C.c_int, [_vp, _i32p, _i32p, _i32p, _i32p]),
+                                    C.c_int32, C.c_int32, C.c_int32, _i32p, _i32p, _i32p, _i32p,
+                                    _i32p]),
+    "kap_schedule_info": (C.c_int, [_vp, _i32p, _i32p, _i32p, _i32p, _i32p]),
     "kap_selected_decode_attn": (C.c_int, [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, C.c_int32,
                                            C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float,
                                            _vp, _vp, _vp, _vp]),
@@ -90,10 +91,10 @@ def launch_count() -> int:
     return int(lib().kap_launch_count())
 
 
-def set_launch_options(use_pdl: int = -1, fused_merge: int = -1, ctas_per_sm: int = -1,
-                       early_kv: int = -1):
-    _check(lib().kap_set_launch_options(int(use_pdl), int(fused_merge), int(ctas_per_sm),
-                                        int(early_kv)))
+def set_launch_options(use_pdl: int = -1, early_kv: int = -1, ctas_per_sm: int = -1,
+                       max_cluster: int = -1):
+    _check(lib().kap_set_launch_options(int(use_pdl), int(early_kv), int(ctas_per_sm),
+                                        int(max_cluster)))
 
 
 # ------------------------------------------------------------------------------- kap_compile_plan
@@ -137,18 +138,21 @@ def compile_workload(w, capacity=None):
 
 
 def schedule_host(list_len, n_q, num_q_heads, num_kv_heads, cta_slots, max_chunk_pages=0,
-                  max_items=8192):
+                  max_items=8192, max_cluster=1):
     """kap_schedule_host: the split-K work list as an [n_items, 8] int32 array (seq, kv_head,
-    page_begin, page_end, group, slot, n_splits, n_q) plus (n_merge_groups, max_chunk)."""
+    page_begin, page_end, group, slot, n_splits, n_q) plus (n_merge_groups, max_chunk) and, when
+    max_cluster > 1, the chosen cluster size as a fourth value."""
     list_len = _np(list_len, np.int32)
     n_q = _np(n_q, np.int32)
     items = np.zeros((max_items, 8), dtype=np.int32)
-    n_items, n_merge, max_chunk = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    n_items, n_merge, max_chunk, cluster = C.c_int32(0), C.c_int32(0), C.c_int32(0), C.c_int32(1)
     _check(lib().kap_schedule_host(int(list_len.shape[0]), _ptr(list_len, C.c_int32),
                                    _ptr(n_q, C.c_int32), num_q_heads, num_kv_heads, cta_slots,
-                                   max_chunk_pages, max_items, _ptr(items, C.c_int32),
-                                   C.byref(n_items), C.byref(n_merge), C.byref(max_chunk)))
-    return items[:n_items.value].copy(), n_merge.value, max_chunk.value
+                                   max_cluster, max_chunk_pages, max_items, _ptr(items, C.c_int32),
+                                   C.byref(n_items), C.byref(n_merge), C.byref(max_chunk),
+                                   C.byref(cluster)))
+    out = (items[:n_items.value].copy(), n_merge.value, max_chunk.value)
+    return out if max_cluster <= 1 else out + (cluster.value,)
 
 
 # ------------------------------------------------------------------------- workspace + attention
@@ -188,10 +192,10 @@ class Workspace:
         return self.info()
 
     def info(self):
-        v = [C.c_int32(0) for _ in range(4)]
+        v = [C.c_int32(0) for _ in range(5)]
         _check(lib().kap_schedule_info(self._h, *[C.byref(x) for x in v]))
         return dict(n_items=v[0].value, n_merge_groups=v[1].value, max_chunk_pages=v[2].value,
-                    ctas_per_wave=v[3].value)
+                    ctas_per_wave=v[3].value, cluster_size=v[4].value)
 
     def check(self, stream=None):
         _check(lib().kap_workspace_check(self._h, _stream_ptr(stream)))

@@ -284,40 +284,60 @@ def test_split_and_launch_option_invariance():
     plan = kap.compile_workload(w)
     qd = _decode_rows(w, q_bits)
     ref = gu.oracle_decode(qd, pool_bits, plan, w.ctx_len)
-    one_split = gu.run_decode(qd, pool, plan, w.ctx_len, max_chunk_pages=512)
+    ref_v = gu.oracle_verify(q_bits, w.n_q, pool_bits, w.bt_indptr, w.bt_pages, w.ctx_len)
     try:
+        kap.set_launch_options(1, 1, -1, 1)
+        one_split = gu.run_decode(qd, pool, plan, w.ctx_len, max_chunk_pages=512)
         for pdl, early in ((0, 0), (1, 0), (1, 1)):
-            for fused in (0, 1):
-                kap.set_launch_options(pdl, fused, -1, early)
+            for cluster in (1, 2, 4, 8):
+                kap.set_launch_options(pdl, early, -1, cluster)
                 for chunk in (0, 1, 7):
                     got = gu.run_decode(qd, pool, plan, w.ctx_len, max_chunk_pages=chunk)
-                    _check_pair(got, ref, f"pdl={pdl} fused={fused} chunk={chunk}")
+                    _check_pair(got, ref, f"pdl={pdl} early={early} cluster={cluster} chunk={chunk}")
                     # splits only reorder fp32 sums: far tighter than the oracle tolerance
                     np.testing.assert_allclose(got[0], one_split[0], atol=2e-3, rtol=1e-2)
                     np.testing.assert_allclose(got[1], one_split[1], atol=1e-4)
                 got = gu.run_verify(q_bits, w.n_q, pool, w.bt_indptr, w.bt_pages, w.ctx_len)
-                _check_pair(got, gu.oracle_verify(q_bits, w.n_q, pool_bits, w.bt_indptr, w.bt_pages, w.ctx_len),
-                            f"verify pdl={pdl} fused={fused}")
+                _check_pair(got, ref_v, f"verify pdl={pdl} early={early} cluster={cluster}")
     finally:
-        kap.set_launch_options(1, 0, -1, 1)
+        kap.set_launch_options(1, 1, 0, 8)
+
+
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+@pytest.mark.parametrize("cps", [1, 2, 0])
+def test_cluster_sizes_on_ragged_batches(cluster, cps):
+    """Every cluster size on ragged batches with all row-tile counts (n_q 1..16), including lists
+    shorter than the cluster (some CTAs of a cluster get no page at all)."""
+    try:
+        kap.set_launch_options(1, 1, cps, cluster)
+        for seed, batch, max_len, nq in ((1, 5, 700, (1, 2, 3, 4)), (3, 3, 6000, (7, 8, 9)),
+                                         (5, 4, 2500, (13, 16)), (6, 6, 40, (1, 2))):
+            w = _ragged_workload(seed, batch, max_len, nq)
+            q_bits, pool_bits, pool = _workload_case(w, seed)
+            plan = kap.compile_workload(w)
+            qd = _decode_rows(w, q_bits)
+            _check_pair(gu.run_decode(qd, pool, plan, w.ctx_len),
+                        gu.oracle_decode(qd, pool_bits, plan, w.ctx_len), f"cluster {cluster} decode {seed}")
+            _check_pair(gu.run_verify(q_bits, w.n_q, pool, w.bt_indptr, w.bt_pages, w.ctx_len),
+                        gu.oracle_verify(q_bits, w.n_q, pool_bits, w.bt_indptr, w.bt_pages, w.ctx_len),
+                        f"cluster {cluster} verify {seed}")
+    finally:
+        kap.set_launch_options(1, 1, 0, 8)
 
 
 def test_repeated_calls_and_workspace_reuse():
-    """One workspace, one schedule, many calls (the per-layer loop); results are identical run to
-    run, and the fused-merge counters are left clean."""
+    """One workspace, one schedule, many calls (the per-layer loop): identical results run to run."""
     w = synth.config2(0, batch=2, L=4096, layers=1)
     q_bits, pool_bits, pool = _workload_case(w, 6)
     plan = kap.compile_workload(w)
     qd = _decode_rows(w, q_bits)
     ws = kap.Workspace(max_rows_per_item=4, max_batch=2)
     try:
-        kap.set_launch_options(1, 1)
         first = gu.run_decode(qd, pool, plan, w.ctx_len, ws=ws, max_chunk_pages=4)
         for _ in range(3):
             again = gu.run_decode(qd, pool, plan, w.ctx_len, ws=ws, max_chunk_pages=4)
             np.testing.assert_array_equal(first[0], again[0])
     finally:
-        kap.set_launch_options(1, 0, -1, 1)
         ws.close()
 
 

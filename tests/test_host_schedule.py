@@ -7,13 +7,13 @@ import pytest
 from paper_2607_24260_b200 import kap, synth
 
 
-def _verify_schedule(list_len, n_q, items, Hkv, cap):
+def _verify_schedule(list_len, n_q, items, Hkv, cap, cluster=1):
     B = len(list_len)
     cover = [[np.zeros(int(list_len[b]), dtype=np.int32) for _ in range(Hkv)] for b in range(B)]
     slots = set()
     by_group = {}
     sizes = items[:, 3] - items[:, 2]
-    assert np.all(sizes >= 1) and np.all(sizes <= cap)
+    assert np.all(sizes >= 1) and np.all(-(-sizes // cluster) <= cap)
     assert np.all(np.diff(sizes) <= 0), "items must be sorted longest first"
     for seq, g, p0, p1, group, slot, n_splits, nq in items.tolist():
         cover[seq][g][p0:p1] += 1
@@ -92,3 +92,25 @@ def test_schedule_errors():
     with pytest.raises(kap.KapError) as e:          # 10 groups cannot fit 4 items
         kap.schedule_host([4] * 10, None, 4, 1, 296, 0, max_items=4)
     assert e.value.code == kap.ERR_CAPACITY
+
+
+def test_cluster_schedules():
+    """With clusters allowed the uniform configurations fit one cluster per (sequence, KV head):
+    no merge pass, and the per-CTA chunk is the cluster's share."""
+    for name, want_cluster in (("c2", 4), ("c3", 2), ("c4", 8)):
+        w = synth.CONFIGS[name](0)
+        n = np.diff(kap.compile_workload(w)["plan_indptr"])
+        items, n_merge, max_chunk, cluster = kap.schedule_host(n, None, 32, 8, 296, max_cluster=8)
+        _verify_schedule(n, None, items, 8, 512, cluster)
+        assert cluster == want_cluster and n_merge == 0 and len(items) == w.batch * 8
+        assert max_chunk == -(-int(n.max()) // cluster)
+    rng = synth.rng_for(1, "sched-cluster")
+    for _ in range(100):
+        B = int(rng.integers(1, 40))
+        n = rng.integers(1, 9000, size=B).astype(np.int32)
+        nq = rng.integers(1, 9, size=B).astype(np.int32) if rng.random() < 0.5 else None
+        mc = int(rng.choice([2, 4, 8]))
+        items, n_merge, max_chunk, cluster = kap.schedule_host(n, nq, 32, 8, int(rng.choice([296, 444])),
+                                                               max_items=100000, max_cluster=mc)
+        assert cluster in (1, 2, 4, 8) and cluster <= mc
+        _verify_schedule(n, nq, items, 8, 512, cluster)
