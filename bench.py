@@ -410,6 +410,7 @@ def main():
     ap.add_argument("--sweep-layers", type=int, default=8)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--max-cluster", type=int, default=-1)
+    ap.add_argument("--ring-slots", type=int, default=-1)
     ap.add_argument("--pdl", type=int, default=-1)
     ap.add_argument("--ctas-per-sm", type=int, default=-1)
     ap.add_argument("--early-kv", type=int, default=-1)
@@ -428,7 +429,7 @@ def main():
     if world > 1:
         from paper_2607_24260_b200 import dist as kdist
         dist = kdist.Group("nccl", device=dev)
-    kap.set_launch_options(args.pdl, args.early_kv, args.ctas_per_sm, args.max_cluster)
+    kap.set_launch_options(args.pdl, args.early_kv, args.ctas_per_sm, args.max_cluster, args.ring_slots)
     warmup = max(3, args.warmup)
 
     cy = Cycle(args.config, seed=rank, layers=args.layers, device=dev)
@@ -456,7 +457,7 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": config_dict(w, k, cy.layers, {"parallelism": f"dp{world} (independent batches per GPU)",
-                                                 "pdl": args.pdl, "max_cluster": args.max_cluster,
+                                                 "pdl": args.pdl, "max_cluster": args.max_cluster, "ring_slots": args.ring_slots,
                                                  "ctas_per_sm": args.ctas_per_sm, "early_kv": args.early_kv}),
         "clocks": clocks.summary(),
         "e2e": {"value": world * w.batch * k / (e2e_ms * 1e-3), "unit": "tokens/s",

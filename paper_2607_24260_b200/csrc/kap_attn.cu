@@ -40,30 +40,32 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
 // ------------------------------------------------------------------------------ kernel geometry
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
-constexpr int kSlots = 8;                                 // page slots in the shared-memory ring
+constexpr int kMaxSlots = 24;                             // most page slots in the shared-memory ring
+constexpr int kDefaultSlots = 8;                          // 8 slots -> 3 CTAs/SM, 12 -> 2, 24 -> 1
 constexpr int kHalfTileBytes = kPageSize * 128;           // 16 tokens x 64 bf16 = 2048 B
 constexpr int kTileBytes = 2 * kHalfTileBytes;            // K (or V) of one page and head: 4096 B
 constexpr int kPageHeadBytes = 2 * kTileBytes;            // K + V: 8192 B
-constexpr int kRingBytes = kSlots * kPageHeadBytes;       // 64 KiB
-constexpr int kMaxChunk = 512;                            // page ids a CTA can hold
+constexpr int kMaxIds = 768;                              // page ids a CTA can hold (dynamic sharing up to this)
 constexpr int kScratchStride = kHeadDim + 8;              // floats per scratch row (bank spread)
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;         // per-CTA deadline for all waits
 
-struct SmemTail {                                         // what follows the ring
-    int32_t phys[kMaxChunk];
-    int32_t logical[kMaxChunk];
-    unsigned long long full[kSlots];
-    unsigned long long empty[kSlots];
+struct SmemTail {                                         // control block in front of the ring
+    int32_t phys[kMaxIds];
+    int32_t logical[kMaxIds];
+    int32_t slot_page[kMaxSlots];             // list index of the page in each ring slot, -1 = no more
+    uint32_t slot_done[kMaxSlots];            // warps that have finished with the slot's current page
+    unsigned long long full[kMaxSlots];
     float m[kWarps][kRowTile];
     float l[kWarps][kRowTile];
     float cta_m[kRowTile * kMaxRowTiles];     // CTA-level state read by cluster peers
     float cta_l[kRowTile * kMaxRowTiles];
     int32_t timed_out;
 };
-constexpr int kSmemBytes = kRingBytes + (int)sizeof(SmemTail) + 1024;   // + alignment slack
+constexpr int kTailBytes = ((int)sizeof(SmemTail) + 1023) / 1024 * 1024;   // the ring follows, 1 KiB aligned
+constexpr int smem_bytes_for(int slots) { return kTailBytes + slots * kPageHeadBytes + 1024; }  // + alignment slack
 
-static_assert(kWarps * kRowTile * kScratchStride * 4 <= kRingBytes,
-              "warp-combine scratch must fit in the ring");
+static_assert(kWarps * kRowTile * kScratchStride * 4 <= kDefaultSlots * kPageHeadBytes,
+              "warp-combine scratch must fit in the smallest ring");
 
 struct AttnParams {
     const __nv_bfloat16* q;          // [rows, Hq, d]
@@ -82,6 +84,7 @@ struct AttnParams {
     long long num_pool_pages;
     int32_t Hq, Hkv, G, rows_cap;
     int32_t cluster, early_kv;       // CTAs per work item (cluster size); early KV prefetch
+    int32_t ring_slots;              // page slots in the shared-memory ring (8, 12, 16 or 24)
     float scale_log2;                // sm_scale * log2(e)
 #ifdef KAP_TRACE
     unsigned long long* trace;       // [8192 records][8] timestamps of this launch (debug builds)
@@ -261,32 +264,37 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
 {
     extern __shared__ unsigned char smem_raw[];
     // the 128-byte swizzle pattern repeats every 1024 bytes: tiles must start on that boundary
-    unsigned char* ring = reinterpret_cast<unsigned char*>(
+    unsigned char* smem_base = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    SmemTail* tail = reinterpret_cast<SmemTail*>(ring + kRingBytes);
+    SmemTail* tail = reinterpret_cast<SmemTail*>(smem_base);
+    unsigned char* ring = smem_base + kTailBytes;
+    const int n_slots = p.ring_slots;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     pdl_launch_dependents();
     KAP_TRACE_POINT(blockIdx.x, 0);
 
     // ---- prologue on static metadata only (work list, page lists, q_indptr): with programmatic
     // dependent launch it overlaps the tail of the previous kernel on the stream.
-    // A work item belongs to a cluster of C CTAs (C = 1: no cluster); CTA `rank` takes its even
-    // share of the item's pages.
+    // A work item belongs to a cluster of C CTAs (C = 1: no cluster).  Its pages are dealt
+    // round-robin to the warp groups: over all groups of all C CTAs when the whole item's id list
+    // fits in shared memory, otherwise every CTA takes an even slice of the item and deals that.
     const int C = p.cluster, rank = blockIdx.x % C;
     WorkItem item = p.items[blockIdx.x / C];
-    {
+    const bool shared_list = (item.page_end - item.page_begin) <= kMaxIds;
+    if (!shared_list) {
         const int n = item.page_end - item.page_begin, base = n / C, rem = n % C;
         item.page_begin += rank * base + min(rank, rem);
         item.page_end = item.page_begin + base + (rank < rem ? 1 : 0);
     }
-    const int n_pages = item.page_end - item.page_begin;
+    if (tid == 0 && item.page_end - item.page_begin > kMaxIds) atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX);
+    const int n_pages = min(item.page_end - item.page_begin, kMaxIds);   // the scheduler caps slices at 512
     const int rows = item.n_q * p.G;                         // valid query rows of this item
     int RT = (rows + kRowTile - 1) / kRowTile;               // row tiles: 1, 2 or 4
     if (RT == 3) RT = 4;
     if (tid == 0) {
-        for (int s = 0; s < kSlots; ++s) {
+        for (int s = 0; s < n_slots; ++s) {
             mbar_init(smem_u32(&tail->full[s]), 1);
-            mbar_init(smem_u32(&tail->empty[s]), RT);
+            tail->slot_done[s] = 0;
         }
         tail->timed_out = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -310,41 +318,48 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     KAP_TRACE_POINT(blockIdx.x, 1);
 
     const int n_groups = kWarps / RT;                        // warp groups
-    const int depth = kSlots / n_groups;                     // ring slots per group
+    const int depth = n_slots / n_groups;                    // ring slots per group
     const int grp = warp / RT, rt = warp % RT;
-    const int n_mine = grp < n_pages ? (n_pages - grp + n_groups - 1) / n_groups : 0;
-    const bool producer = (rt == 0) && (lane == 0);
+    const bool producer = (rt == 0) && (lane == 0);           // fills the group's ring at the start
     const int rows_per_page = 2 * p.Hkv * kPageSize;
     const int v_row_off = p.Hkv * kPageSize;
-    uint64_t policy = 0;
-    if (producer) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-
-    // issue the loads of this group's i-th page into ring slot grp * depth + i % depth
-    auto issue = [&](int i) {
-        const int s = grp * depth + i % depth;
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    // the k-th page of this warp group is list entry first_idx + k * idx_stride
+    const int idx_stride = (shared_list ? C : 1) * n_groups;
+    const int first_idx = (shared_list ? rank : 0) * n_groups + grp;
+    // put the group's k-th page into ring slot s, or publish "no more pages" there
+    auto fill = [&](int s, int k) {
         const uint32_t bar = smem_u32(&tail->full[s]);
-        const int y = tail->phys[grp + i * n_groups] * rows_per_page + item.kv_head * kPageSize;
-        const uint32_t dst = smem_u32(ring + s * kPageHeadBytes);
-        mbar_expect_tx(bar, kPageHeadBytes);
-        tma_load_2d(dst, &kv_map, 0, y, bar, policy);
-        tma_load_2d(dst + kHalfTileBytes, &kv_map, 64, y, bar, policy);
-        tma_load_2d(dst + kTileBytes, &kv_map, 0, y + v_row_off, bar, policy);
-        tma_load_2d(dst + kTileBytes + kHalfTileBytes, &kv_map, 64, y + v_row_off, bar, policy);
+        const int idx = first_idx + k * idx_stride;
+        if (idx < n_pages) {
+            tail->slot_page[s] = idx;
+            const int y = tail->phys[idx] * rows_per_page + item.kv_head * kPageSize;
+            const uint32_t dst = smem_u32(ring + s * kPageHeadBytes);
+            mbar_expect_tx(bar, kPageHeadBytes);
+            tma_load_2d(dst, &kv_map, 0, y, bar, policy);
+            tma_load_2d(dst + kHalfTileBytes, &kv_map, 64, y, bar, policy);
+            tma_load_2d(dst + kTileBytes, &kv_map, 0, y + v_row_off, bar, policy);
+            tma_load_2d(dst + kTileBytes + kHalfTileBytes, &kv_map, 64, y + v_row_off, bar, policy);
+        } else {
+            tail->slot_page[s] = -1;
+            mbar_arrive(bar);                                // completes the phase with no bytes
+        }
     };
     // Early KV prefetch: pages that hold only tokens older than the query rows' own tokens
     // (t < L - n_q) were written in earlier steps, so their loads may start before the previous
     // kernel on the stream has completed.  Pages holding the rows' own tokens, Q and the partial
     // buffers wait for it.  (ctx_len must then be final before the previous kernel was launched.)
-    const int first = min(depth, n_mine);
-    int issued = 0, L = 0;
+    int filled = 0, L = 0;
     if (p.early_kv) {
         L = p.ctx_len[item.seq];
         if (producer) {
             const int fresh_from = L - item.n_q;
-            while (issued < first &&
-                   tail->logical[grp + issued * n_groups] * kPageSize + kPageSize - 1 < fresh_from) {
-                issue(issued);
-                ++issued;
+            while (filled < depth) {
+                const int idx = first_idx + filled * idx_stride;
+                if (idx >= n_pages || tail->logical[idx] * kPageSize + kPageSize - 1 >= fresh_from) break;
+                fill(grp * depth + filled, filled);
+                ++filled;
             }
         }
     }
@@ -352,7 +367,7 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     pdl_wait();
     KAP_TRACE_POINT(blockIdx.x, 2);
     if (producer)
-        for (; issued < first; ++issued) issue(issued);
+        for (; filled < depth; ++filled) fill(grp * depth + filled, filled);
     if (!p.early_kv) L = p.ctx_len[item.seq];
     const uint64_t deadline = global_ns() + kWaitBudgetNs;
 
@@ -390,14 +405,16 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     const int k_tok = ((lm >> 1) << 3) + lr, k_cbit = lm & 1;   // K: matrices (n-tile, k-half)
     const int v_tok = ((lm & 1) << 3) + lr, v_cbit = lm >> 1;   // V^T: matrices (k-half, n-tile)
 
-    for (int i = 0; i < n_mine; ++i) {
+    for (int i = 0;; ++i) {
         const int s = grp * depth + i % depth;
         const uint32_t parity = (i / depth) & 1;
         mbar_wait(smem_u32(&tail->full[s]), parity, deadline, &tail->timed_out);
         if (i == 0) KAP_TRACE_POINT(blockIdx.x, 3);
+        const int page = tail->slot_page[s];
+        if (page < 0 || tail->timed_out) break;              // the list is exhausted
         const uint32_t kb = smem_u32(ring + s * kPageHeadBytes);
         const uint32_t vb = kb + kTileBytes;
-        const int tok0 = tail->logical[grp + i * n_groups] * kPageSize;
+        const int tok0 = tail->logical[page] * kPageSize;
 
         // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
         float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -471,12 +488,21 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             mma_bf16(o[2 * n2], pa, v0, v1);
             mma_bf16(o[2 * n2 + 1], pa, v2, v3);
         }
-        // release the slot; the group's producer lane refills it once all RT warps have
+        // Done with the slot.  The last of the group's RT warps to get here refills it with the
+        // group's page i + depth; nobody waits for anybody.  The fences order this warp's reads
+        // of the slot before the counter update and the refill's asynchronous writes after it.
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tail->empty[s]));
-        if (producer && i + depth < n_mine) {
-            mbar_wait(smem_u32(&tail->empty[s]), parity, deadline, &tail->timed_out);
-            issue(i + depth);
+        if (lane == 0) {
+            bool last = true;
+            if (RT > 1) {
+                __threadfence_block();
+                last = atomicAdd(&tail->slot_done[s], 1u) == (uint32_t)(RT - 1);
+                if (last) { tail->slot_done[s] = 0; __threadfence_block(); }
+            }
+            if (last) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                fill(s, i + depth);
+            }
         }
     }
     if (lane == 0 && tail->timed_out) atomicOr(p.status, 1 << KAP_ERR_TIMEOUT);
@@ -593,6 +619,7 @@ std::atomic<long long> g_launches{0};
 std::atomic<int> g_use_pdl{1};
 std::atomic<int> g_max_cluster{8};       // largest thread-block cluster the scheduler may pick
 std::atomic<int> g_early_kv{1};
+std::atomic<int> g_ring_slots{kDefaultSlots};
 std::atomic<int> g_ctas_per_sm{0};       // 0 = as many as fit (occupancy)
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -667,13 +694,15 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     if (st != KAP_OK) return st;
     std::call_once(g_attr_once, [] {
         g_attr_err = cudaFuncSetAttribute(kap_attn_split_kernel,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          smem_bytes_for(kMaxSlots));
     });
     if (g_attr_err != cudaSuccess)
         return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(g_attr_err));
 
     AttnParams p = p_in;
     p.cluster = ws->cluster_size;
+    p.ring_slots = ws->ring_slots;
     p.early_kv = (g_use_pdl.load() && g_early_kv.load()) ? 1 : 0;
 #ifdef KAP_TRACE
     p.trace = (g_trace && g_trace_next < g_trace_cap) ? g_trace + (size_t)(g_trace_next++) * 8192 * 8 : nullptr;
@@ -696,7 +725,7 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)ws->n_items * (unsigned)ws->cluster_size);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.dynamicSmemBytes = smem_bytes_for(ws->ring_slots);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
@@ -777,29 +806,6 @@ extern "C" kap_status kap_workspace_create(kap_workspace** out, int32_t device, 
         kap_workspace_destroy(ws);
         return fail(KAP_ERR_CUDA, "workspace allocation failed: %s", cudaGetErrorString(e));
     }
-    // resident CTAs per SM decide how many items make one wave
-    int per_sm = 0;
-    cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kap_attn_split_kernel, kThreads,
-                                                      kSmemBytes) != cudaSuccess || per_sm < 1)
-        per_sm = 1;
-    ws->occupancy = per_sm;
-    ws->ctas_per_wave = per_sm * ws->sm_count;
-    // how many clusters of 2, 4, 8 CTAs can be resident at once (GPC boundaries cost a few)
-    for (int ci = 1; ci < 4; ++ci) {
-        cudaLaunchAttribute ca[1];
-        ca[0].id = cudaLaunchAttributeClusterDimension;
-        ca[0].val.clusterDim.x = 1u << ci; ca[0].val.clusterDim.y = 1; ca[0].val.clusterDim.z = 1;
-        cudaLaunchConfig_t cc{};
-        cc.gridDim = dim3((unsigned)(ws->sm_count * per_sm / (1 << ci)) * (1u << ci));
-        cc.blockDim = dim3(kThreads);
-        cc.dynamicSmemBytes = kSmemBytes;
-        cc.attrs = ca; cc.numAttrs = 1;
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
-        ws->max_clusters[ci] = n;
-    }
-    ws->max_clusters[0] = ws->ctas_per_wave;
     *out = ws;
     return KAP_OK;
 }
@@ -823,17 +829,37 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     std::vector<WorkItem> items;
     std::vector<MergeGroup> groups;
     int32_t max_chunk = 0, row_tiles = 1;
-    // resident slots per cluster size: all of the SM's CTA slots, or ctas_per_sm of them
+    // resident CTAs per SM for the chosen ring size decide how many items make one wave;
+    // clusters of 2, 4, 8 CTAs fit a few less (GPC boundaries)
+    KAP_CUDA(cudaSetDevice(ws->device));
+    const int ring_slots = g_ring_slots.load();
+    const int smem = smem_bytes_for(ring_slots);
+    cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         smem_bytes_for(kMaxSlots));
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel, kThreads, smem) != cudaSuccess || occ < 1)
+        occ = 1;
     const int want = g_ctas_per_sm.load();
-    const int per_sm = want > 0 ? std::min(want, ws->occupancy) : ws->occupancy;
+    const int per_sm = want > 0 ? std::min(want, occ) : occ;
+    ws->occupancy = occ;
+    ws->ring_slots = ring_slots;
     ws->ctas_per_wave = per_sm * ws->sm_count;
-    int32_t slots[4];
-    for (int ci = 0; ci < 4; ++ci) {
+    int32_t slots[4] = {ws->ctas_per_wave, 0, 0, 0};
+    for (int ci = 1; ci < 4; ++ci) {
         const int c = 1 << ci;
-        const int64_t scaled = (int64_t)ws->max_clusters[ci] * per_sm / ws->occupancy;
-        slots[ci] = c <= g_max_cluster.load() ? (int32_t)std::min<int64_t>(scaled, ws->ctas_per_wave / c) : 0;
+        if (c > g_max_cluster.load()) continue;
+        cudaLaunchAttribute ca[1];
+        ca[0].id = cudaLaunchAttributeClusterDimension;
+        ca[0].val.clusterDim.x = (unsigned)c; ca[0].val.clusterDim.y = 1; ca[0].val.clusterDim.z = 1;
+        cudaLaunchConfig_t cc{};
+        cc.gridDim = dim3((unsigned)(ws->sm_count * occ / c) * (unsigned)c);
+        cc.blockDim = dim3(kThreads);
+        cc.dynamicSmemBytes = smem;
+        cc.attrs = ca; cc.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
+        slots[ci] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
     }
-    slots[0] = ws->ctas_per_wave;
     int32_t cluster = 1;
     kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots,
                                    max_chunk_pages, ws->max_items, ws->max_rows, items, groups,
@@ -945,7 +971,10 @@ extern "C" kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream) 
 }
 
 extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, int32_t ctas_per_sm,
-                                             int32_t max_cluster) {
+                                             int32_t max_cluster, int32_t ring_slots) {
+    if (ring_slots >= 0 && ring_slots != 8 && ring_slots != 12 && ring_slots != 16 && ring_slots != 24)
+        return fail(KAP_ERR_INVALID_ARG, "ring_slots %d (allowed: 8, 12, 16, 24)", ring_slots);
+    if (ring_slots > 0) g_ring_slots.store(ring_slots);
     if (max_cluster == 0 || max_cluster > 8 || (max_cluster > 0 && (max_cluster & (max_cluster - 1))))
         return fail(KAP_ERR_INVALID_ARG, "max_cluster %d (allowed: 1, 2, 4, 8)", max_cluster);
     if (use_pdl >= 0) g_use_pdl.store(use_pdl ? 1 : 0);
@@ -1069,7 +1098,8 @@ extern "C" kap_status kap_selected_decode_attn_static(
             void* ptr = nullptr;
             KAP_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
             KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          smem_bytes_for(kMaxSlots)));
             g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
             g_static_ready[dev] = true;
         }
@@ -1104,7 +1134,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
     p.out = (__nv_bfloat16*)out; p.lse = lse;
     p.status = reinterpret_cast<int32_t*>(base);
     p.num_pool_pages = num_pool_pages; p.Hq = num_q_heads; p.Hkv = num_kv_heads; p.G = rows;
-    p.rows_cap = rows; p.cluster = 1; p.early_kv = 0;
+    p.rows_cap = rows; p.cluster = 1; p.early_kv = 0; p.ring_slots = kDefaultSlots;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
 #ifdef KAP_TRACE
     p.trace = nullptr;
@@ -1122,7 +1152,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
     g_launches.fetch_add(1);
     // plain launches: the work list was written by the kernel just before, so the split kernel
     // must not start early
-    kap_attn_split_kernel<<<(unsigned)n_items, kThreads, kSmemBytes, stream>>>(map, p);
+    kap_attn_split_kernel<<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
     KAP_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     if (num_splits > 1) {

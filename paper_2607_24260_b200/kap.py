@@ -40,7 +40,7 @@ SIGNATURES = {
                                                   C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                   C.c_float, C.c_int32, _vp, _vp, _vp, _vp]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
-    "kap_set_launch_options": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
+    "kap_set_launch_options": (C.c_int, [C.c_int32] * 5),
     "kap_launch_count": (C.c_int64, []),
     "kap_last_error": (C.c_char_p, []),
     "kap_version": (C.c_char_p, []),
@@ -92,9 +92,9 @@ def launch_count() -> int:
 
 
 def set_launch_options(use_pdl: int = -1, early_kv: int = -1, ctas_per_sm: int = -1,
-                       max_cluster: int = -1):
+                       max_cluster: int = -1, ring_slots: int = -1):
     _check(lib().kap_set_launch_options(int(use_pdl), int(early_kv), int(ctas_per_sm),
-                                        int(max_cluster)))
+                                        int(max_cluster), int(ring_slots)))
 
 
 # ------------------------------------------------------------------------------- kap_compile_plan

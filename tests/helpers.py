@@ -39,3 +39,14 @@ def assert_close(got, ref, atol=ATOL, rtol=RTOL, what=""):
         i = np.unravel_index(np.argmax(np.where(bad, err - bound, -np.inf)), err.shape)
         raise AssertionError(f"{what}: {bad.sum()} of {bad.size} outside |d|<={atol}+{rtol}|ref|; "
                              f"worst at {i}: got {got[i]!r} ref {ref[i]!r}")
+
+
+def assert_same_up_to_rounding(a, b, what=""):
+    """Two runs of the library on inputs whose differences must not matter: equal up to the order
+    of the fp32 sums, i.e. within two bf16 ulps of the largest magnitude (pages are handed out
+    dynamically, so the summation order is not fixed)."""
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    scale = max(float(np.max(np.abs(b))), 1e-30)
+    err = float(np.max(np.abs(a - b)))
+    assert err <= 2.0 ** -7 * scale, f"{what}: max diff {err} vs scale {scale}"

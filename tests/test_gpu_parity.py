@@ -7,7 +7,7 @@ import pytest
 import torch
 
 import gpu_util as gu
-from helpers import ATOL, RTOL, assert_close
+from helpers import ATOL, RTOL, assert_close, assert_same_up_to_rounding
 from oracle import kap_oracle as orc
 from paper_2607_24260_b200 import kap, synth
 
@@ -219,12 +219,12 @@ def test_probe_one_hot_key_and_invisible_key():
     np.testing.assert_allclose(out[0, head], v, atol=1e-6)           # the weight is 1 to ~e-30
     assert abs(lse[0, head] - 40.0) < 0.3
     others = [h for h in range(32) if h // 4 != head // 4]
-    np.testing.assert_array_equal(out[0, others], base[0, others])
+    assert_same_up_to_rounding(out[0, others], base[0, others], "other heads")
     pool = pool_bits.copy()
     _plant(pool, w, hidden * 16 + 5, qd[0], head)
     out2, lse2 = gu.run_decode(qd, gu.bits_to_dev(pool), plan, w.ctx_len)
-    np.testing.assert_array_equal(out2, base)
-    np.testing.assert_array_equal(lse2, base_lse)
+    assert_same_up_to_rounding(out2, base, "invisible key")
+    np.testing.assert_allclose(lse2, base_lse, atol=1e-5)
 
 
 @pytest.mark.parametrize("nq", [4, 8, 7])
@@ -243,7 +243,7 @@ def test_probe_verify_causality(nq):
     v = synth.bf16_bits_to_f64(pool[w.bt_pages[lp], 1, head // 4, s])
     for r in range(nq):
         if r <= j:
-            np.testing.assert_array_equal(out[r, head], base[r, head])
+            assert_same_up_to_rounding(out[r, head], base[r, head], f"row {r}")
         else:
             np.testing.assert_allclose(out[r, head], v, atol=1e-6)
 
@@ -257,7 +257,7 @@ def test_verify_last_row_equals_identity_plan_decode():
                  plan_phys_pages=w.bt_pages[:n_pages].astype(np.int32))
     d_out, d_lse = gu.run_decode(q_bits[7:8], pool, ident, w.ctx_len)
     d2_out, d2_lse = gu.run_decode(q_bits[7:8], pool, ident, w.ctx_len, logical=False)
-    np.testing.assert_array_equal(d_out, d2_out)          # NULL logical list == identity positions
+    assert_same_up_to_rounding(d_out, d2_out, "NULL logical list == identity positions")
     np.testing.assert_allclose(v_out[7], d_out[0], atol=2e-3, rtol=1e-2)
     np.testing.assert_allclose(v_lse[7], d_lse[0], atol=1e-4)
 
@@ -270,11 +270,11 @@ def test_garbage_beyond_context_is_ignored():
     dirty_bits = pool_bits.copy()
     dirty_bits[w.bt_pages[n_pages - 1], :, :, L % 16:, :] = 0x7FC0     # NaN
     dirty = gu.run_decode(q_bits[:1], gu.bits_to_dev(dirty_bits), plan, w.ctx_len)
-    np.testing.assert_array_equal(clean[0], dirty[0])
-    np.testing.assert_array_equal(clean[1], dirty[1])
+    assert_same_up_to_rounding(clean[0], dirty[0], "decode with NaN tail")
+    np.testing.assert_allclose(clean[1], dirty[1], atol=1e-5)
     v_clean = gu.run_verify(q_bits[:4], [4], gu.bits_to_dev(pool_bits), w.bt_indptr, w.bt_pages, w.ctx_len)
     v_dirty = gu.run_verify(q_bits[:4], [4], gu.bits_to_dev(dirty_bits), w.bt_indptr, w.bt_pages, w.ctx_len)
-    np.testing.assert_array_equal(v_clean[0], v_dirty[0])
+    assert_same_up_to_rounding(v_clean[0], v_dirty[0], "verify with NaN tail")
 
 
 # ------------------------------------------------------------- split / launch-option invariance
@@ -300,16 +300,16 @@ def test_split_and_launch_option_invariance():
                 got = gu.run_verify(q_bits, w.n_q, pool, w.bt_indptr, w.bt_pages, w.ctx_len)
                 _check_pair(got, ref_v, f"verify pdl={pdl} early={early} cluster={cluster}")
     finally:
-        kap.set_launch_options(1, 1, 0, 8)
+        kap.set_launch_options(1, 1, 0, 8, 8)
 
 
 @pytest.mark.parametrize("cluster", [1, 2, 4, 8])
-@pytest.mark.parametrize("cps", [1, 2, 0])
-def test_cluster_sizes_on_ragged_batches(cluster, cps):
+@pytest.mark.parametrize("cps,ring", [(1, 8), (2, 12), (0, 24), (0, 8)])
+def test_cluster_sizes_on_ragged_batches(cluster, cps, ring):
     """Every cluster size on ragged batches with all row-tile counts (n_q 1..16), including lists
     shorter than the cluster (some CTAs of a cluster get no page at all)."""
     try:
-        kap.set_launch_options(1, 1, cps, cluster)
+        kap.set_launch_options(1, 1, cps, cluster, ring)
         for seed, batch, max_len, nq in ((1, 5, 700, (1, 2, 3, 4)), (3, 3, 6000, (7, 8, 9)),
                                          (5, 4, 2500, (13, 16)), (6, 6, 40, (1, 2))):
             w = _ragged_workload(seed, batch, max_len, nq)
@@ -322,11 +322,12 @@ def test_cluster_sizes_on_ragged_batches(cluster, cps):
                         gu.oracle_verify(q_bits, w.n_q, pool_bits, w.bt_indptr, w.bt_pages, w.ctx_len),
                         f"cluster {cluster} verify {seed}")
     finally:
-        kap.set_launch_options(1, 1, 0, 8)
+        kap.set_launch_options(1, 1, 0, 8, 8)
 
 
 def test_repeated_calls_and_workspace_reuse():
-    """One workspace, one schedule, many calls (the per-layer loop): identical results run to run."""
+    """One workspace, one schedule, many calls (the per-layer loop): pages are dealt to warps in a
+    fixed order, so results are bit-identical run to run."""
     w = synth.config2(0, batch=2, L=4096, layers=1)
     q_bits, pool_bits, pool = _workload_case(w, 6)
     plan = kap.compile_workload(w)
@@ -337,6 +338,7 @@ def test_repeated_calls_and_workspace_reuse():
         for _ in range(3):
             again = gu.run_decode(qd, pool, plan, w.ctx_len, ws=ws, max_chunk_pages=4)
             np.testing.assert_array_equal(first[0], again[0])
+            np.testing.assert_array_equal(first[1], again[1])
     finally:
         ws.close()
 
