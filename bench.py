@@ -118,7 +118,7 @@ class ClockSampler:
 class Cycle:
     """Device-resident state of one configuration plus the graphs that replay a cycle."""
 
-    def __init__(self, name, seed, layers=None, device="cuda:0"):
+    def __init__(self, name, seed, layers=None, device="cuda:0", decode_chunk=0, verify_chunk=0):
         import torch
         from paper_2607_24260_b200 import kap, synth
         self.torch, self.kap, self.synth = torch, kap, synth
@@ -155,8 +155,9 @@ class Cycle:
         max_rows = int(w.n_q.max()) * (Hq // Hkv)
         self.ws_d = kap.Workspace(int(device.split(":")[1]), 8192, Hq // Hkv, B)
         self.ws_v = kap.Workspace(int(device.split(":")[1]), 8192, max_rows, B)
-        self.info_d = self.ws_d.schedule(self.n_sel, None, Hq, Hkv)
-        self.info_v = self.ws_v.schedule(self.n_pages, w.n_q, Hq, Hkv)
+        self.info_d = self.ws_d.schedule(self.n_sel, None, Hq, Hkv, decode_chunk)
+        self.info_v = self.ws_v.schedule(self.n_pages, w.n_q, Hq, Hkv, verify_chunk)
+        self.chunks = (decode_chunk, verify_chunk)
         self.graph_d = self.graph_v = None
         self.launches_per_step = 0
 
@@ -285,8 +286,8 @@ def time_e2e(cy: Cycle, steps, warmup):
         h_indptr.numpy()[:] = plan["plan_indptr"]
         h_phys.numpy()[:n] = plan["plan_phys_pages"]
         h_logical.numpy()[:n] = plan["plan_logical_pages"]
-        cy.ws_d.schedule(np.diff(plan["plan_indptr"]), None, w.num_q_heads, w.num_kv_heads)
-        cy.ws_v.schedule(cy.n_pages, w.n_q, w.num_q_heads, w.num_kv_heads)
+        cy.ws_d.schedule(np.diff(plan["plan_indptr"]), None, w.num_q_heads, w.num_kv_heads, cy.chunks[0])
+        cy.ws_v.schedule(cy.n_pages, w.n_q, w.num_q_heads, w.num_kv_heads, cy.chunks[1])
         cy.d_plan_indptr.copy_(h_indptr, non_blocking=True)
         cy.d_plan_phys[:n].copy_(h_phys[:n], non_blocking=True)
         cy.d_plan_logical[:n].copy_(h_logical[:n], non_blocking=True)
@@ -401,7 +402,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
@@ -411,6 +412,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--max-cluster", type=int, default=-1)
     ap.add_argument("--ring-slots", type=int, default=-1)
+    ap.add_argument("--decode-chunk", type=int, default=0, help="cap on pages per CTA, proposal path")
+    ap.add_argument("--verify-chunk", type=int, default=0, help="cap on pages per CTA, verification")
     ap.add_argument("--pdl", type=int, default=-1)
     ap.add_argument("--ctas-per-sm", type=int, default=-1)
     ap.add_argument("--early-kv", type=int, default=-1)
@@ -432,7 +435,8 @@ def main():
     kap.set_launch_options(args.pdl, args.early_kv, args.ctas_per_sm, args.max_cluster, args.ring_slots)
     warmup = max(3, args.warmup)
 
-    cy = Cycle(args.config, seed=rank, layers=args.layers, device=dev)
+    cy = Cycle(args.config, seed=rank, layers=args.layers, device=dev, decode_chunk=args.decode_chunk,
+               verify_chunk=args.verify_chunk)
     cy.capture()
     if dist:
         dist.barrier()
@@ -475,12 +479,14 @@ def main():
 
     if rank == 0 and world == 1 and not args.no_sweep and args.config == "c2":
         sweep = {}
-        for name in ("c3", "c4"):
+        for name in ("c3", "c4", "c5"):
             try:
-                c2 = Cycle(name, seed=0, layers=args.sweep_layers, device=dev)
+                c2 = Cycle(name, seed=0, layers=args.sweep_layers if name != "c5" else max(1, args.sweep_layers // 2),
+                           device=dev)
                 c2.capture()
-                t, d, v = c2.time_steps(max(5, args.steps // 4), 3)
-                r = summarise(c2, max(5, args.steps // 4), t, d, v)
+                n_side = max(5, min(40, args.steps // 4))
+                t, d, v = c2.time_steps(n_side, 3)
+                r = summarise(c2, n_side, t, d, v)
                 sweep[name] = {"workload": c2.w.note, "layers_timed": c2.layers,
                                "us_per_layer_decode": r["us_per_layer_decode"],
                                "us_per_layer_verify": r["us_per_layer_verify"],

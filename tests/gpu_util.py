@@ -13,7 +13,7 @@ DEV = "cuda:0"
 
 def bits_to_dev(bits: np.ndarray) -> torch.Tensor:
     """uint16 bf16 bit patterns -> torch bf16 tensor on the GPU (bit-exact)."""
-    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(DEV).view(torch.bfloat16)
+    return torch.from_numpy(np.array(bits, copy=True).view(np.int16)).to(DEV).view(torch.bfloat16)
 
 
 def dev_to_bits(t: torch.Tensor) -> np.ndarray:
@@ -25,7 +25,7 @@ def dev_bf16_to_f64(t: torch.Tensor) -> np.ndarray:
 
 
 def i32(a) -> torch.Tensor:
-    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(DEV)
+    return torch.from_numpy(np.array(a, dtype=np.int32, copy=True)).to(DEV)
 
 
 def run_decode(q_bits, pool_dev, plan, ctx_len, Hq=32, Hkv=8, max_chunk_pages=0, ws=None,
