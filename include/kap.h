@@ -284,14 +284,14 @@ kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);
  *                pages must then be final before the previous kernel was launched; Q, the pages
  *                holding the rows' own tokens, out and lse may still be written by it.
  *   ctas_per_sm  resident CTAs per SM the scheduler fills in one wave; 0 = as many as fit.
- *   max_cluster  largest thread-block cluster (1, 2, 4 or 8; default 8) the scheduler may give a
- *                work item.  The CTAs of a cluster share the item's pages and reduce their partial
+ *   max_cluster  largest thread-block cluster (1 .. 16; default 16, sizes above 8 use the
+ *                non-portable cluster launch) the scheduler may give a work item.  The CTAs of a cluster share the item's pages and reduce their partial
  *                results through distributed shared memory, so a (sequence, KV head) that fits one
  *                cluster needs no merge pass.
  *   ring_slots   page slots (8 KiB each) in a CTA's shared-memory ring: 8 (3 CTAs per SM), 12 or 16
  *                (2 per SM) or 24 (1 per SM); more slots = more loads in flight per CTA.
  * ctas_per_sm, max_cluster and ring_slots take effect at the next kap_schedule.  The paper has no
- * counterpart for these.  Error: KAP_ERR_INVALID_ARG for a max_cluster that is not 1, 2, 4 or 8 or
+ * counterpart for these.  Error: KAP_ERR_INVALID_ARG for a max_cluster outside 1 .. 16 or
  * a ring_slots that is not 8, 12, 16 or 24. */
 kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, int32_t ctas_per_sm,
                                   int32_t max_cluster, int32_t ring_slots);

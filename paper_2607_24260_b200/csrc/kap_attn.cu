@@ -32,7 +32,7 @@
 namespace kap {
 
 kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t* n_q,
-                          int32_t num_q_heads, int32_t num_kv_heads, const int32_t cluster_slots[4],
+                          int32_t num_q_heads, int32_t num_kv_heads, const int32_t cluster_slots[kMaxCluster],
                           int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
                           std::vector<WorkItem>& items, std::vector<MergeGroup>& groups,
                           int32_t* max_chunk_out, int32_t* row_tiles_out, int32_t* cluster_out);
@@ -233,7 +233,7 @@ __device__ __forceinline__ void store_final(const AttnParams& p, int64_t q_row, 
 // partials are read in batches of independent loads: one memory round trip per batch.
 __device__ __forceinline__ void merge_group_cell(const AttnParams& p, const MergeGroup& g,
                                                  int64_t q_row0, int R, int c4) {
-    constexpr int kBatch = 8;
+    constexpr int kBatch = 16;
     const int64_t base = (int64_t)g.first_item * p.rows_cap + R;
     const int64_t stride = p.rows_cap;
     Merged r; r.m = -INFINITY; r.l = 0.f; r.o = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -617,7 +617,7 @@ namespace {
 
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_use_pdl{1};
-std::atomic<int> g_max_cluster{8};       // largest thread-block cluster the scheduler may pick
+std::atomic<int> g_max_cluster{kMaxCluster};       // largest thread-block cluster the scheduler may pick
 std::atomic<int> g_early_kv{1};
 std::atomic<int> g_ring_slots{kDefaultSlots};
 std::atomic<int> g_ctas_per_sm{0};       // 0 = as many as fit (occupancy)
@@ -696,6 +696,8 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
         g_attr_err = cudaFuncSetAttribute(kap_attn_split_kernel,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           smem_bytes_for(kMaxSlots));
+        cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        cudaGetLastError();
     });
     if (g_attr_err != cudaSuccess)
         return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(g_attr_err));
@@ -844,9 +846,10 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     ws->occupancy = occ;
     ws->ring_slots = ring_slots;
     ws->ctas_per_wave = per_sm * ws->sm_count;
-    int32_t slots[4] = {ws->ctas_per_wave, 0, 0, 0};
-    for (int ci = 1; ci < 4; ++ci) {
-        const int c = 1 << ci;
+    int32_t slots[kMaxCluster] = {ws->ctas_per_wave};
+    cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    cudaGetLastError();
+    for (int c = 2; c <= kMaxCluster; ++c) {
         if (c > g_max_cluster.load()) continue;
         cudaLaunchAttribute ca[1];
         ca[0].id = cudaLaunchAttributeClusterDimension;
@@ -858,7 +861,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         cc.attrs = ca; cc.numAttrs = 1;
         int n = 0;
         if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
-        slots[ci] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
+        slots[c - 1] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
     }
     int32_t cluster = 1;
     kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots,
@@ -975,8 +978,8 @@ extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, 
     if (ring_slots >= 0 && ring_slots != 8 && ring_slots != 12 && ring_slots != 16 && ring_slots != 24)
         return fail(KAP_ERR_INVALID_ARG, "ring_slots %d (allowed: 8, 12, 16, 24)", ring_slots);
     if (ring_slots > 0) g_ring_slots.store(ring_slots);
-    if (max_cluster == 0 || max_cluster > 8 || (max_cluster > 0 && (max_cluster & (max_cluster - 1))))
-        return fail(KAP_ERR_INVALID_ARG, "max_cluster %d (allowed: 1, 2, 4, 8)", max_cluster);
+    if (max_cluster == 0 || max_cluster > kMaxCluster)
+        return fail(KAP_ERR_INVALID_ARG, "max_cluster %d (allowed: 1 .. %d)", max_cluster, kMaxCluster);
     if (use_pdl >= 0) g_use_pdl.store(use_pdl ? 1 : 0);
     if (early_kv >= 0) g_early_kv.store(early_kv ? 1 : 0);
     if (ctas_per_sm >= 0) g_ctas_per_sm.store(ctas_per_sm);

@@ -15,6 +15,7 @@ constexpr int kHeadDim = 128;    // d
 constexpr int kPageSize = 16;    // P
 constexpr int kRowTile = 16;     // query rows one warp carries (one MMA M tile)
 constexpr int kMaxRowTiles = 4;  // => at most 64 rows per (sequence, KV head)
+constexpr int kMaxCluster = 16;  // largest thread-block cluster (sizes above 8 are non-portable)
 
 // One CTA's share of the work: a contiguous slice of one sequence's page list for one KV head.
 struct WorkItem {

@@ -35,9 +35,9 @@ constexpr int64_t kMergePassPages = 9;
 constexpr int64_t kClusterPages = 1;
 constexpr int32_t kDefaultChunkCap = 512;     // per CTA; also the size of the kernel's page-id buffer
 
-// cluster_slots[i] = clusters of size 1 << i that can be resident at once (0 = size not allowed)
+// cluster_slots[c - 1] = clusters of c CTAs that can be resident at once (0 = size not allowed)
 kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t* n_q,
-                          int32_t num_q_heads, int32_t num_kv_heads, const int32_t cluster_slots[4],
+                          int32_t num_q_heads, int32_t num_kv_heads, const int32_t cluster_slots[kMaxCluster],
                           int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
                           std::vector<WorkItem>& items, std::vector<MergeGroup>& groups,
                           int32_t* max_chunk_out, int32_t* row_tiles_out, int32_t* cluster_out)
@@ -83,8 +83,8 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
     int64_t best_t = -1, best_cost = INT64_MAX;
     int32_t best_c = 1;
     const int64_t item_cap = std::max<int64_t>(1, max_items);
-    for (int ci = 0; ci < 4; ++ci) {
-        const int64_t C = 1 << ci;
+    for (int ci = 0; ci < kMaxCluster; ++ci) {
+        const int64_t C = ci + 1;
         if (cluster_slots[ci] <= 0) continue;
         auto consider = [&](int64_t t, int64_t waves) {
             if (t <= 0 || (t + C - 1) / C > cap) return false;
@@ -158,8 +158,8 @@ extern "C" kap_status kap_schedule_host(
     std::vector<kap::WorkItem> items;
     std::vector<kap::MergeGroup> groups;
     int32_t mc = 0, rt = 1, cl = 1;
-    int32_t slots[4];
-    for (int i = 0; i < 4; ++i) slots[i] = (1 << i) <= std::max(max_cluster, 1) ? cta_slots / (1 << i) : 0;
+    int32_t slots[kap::kMaxCluster];
+    for (int i = 0; i < kap::kMaxCluster; ++i) slots[i] = (i + 1) <= std::max(max_cluster, 1) ? cta_slots / (i + 1) : 0;
     kap_status st = kap::build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots,
                                         max_chunk_pages, max_items, kap::kRowTile * kap::kMaxRowTiles,
                                         items, groups, &mc, &rt, &cl);

@@ -289,7 +289,7 @@ def test_split_and_launch_option_invariance():
         kap.set_launch_options(1, 1, -1, 1)
         one_split = gu.run_decode(qd, pool, plan, w.ctx_len, max_chunk_pages=512)
         for pdl, early in ((0, 0), (1, 0), (1, 1)):
-            for cluster in (1, 2, 4, 8):
+            for cluster in (1, 2, 3, 8, 16):
                 kap.set_launch_options(pdl, early, -1, cluster)
                 for chunk in (0, 1, 7):
                     got = gu.run_decode(qd, pool, plan, w.ctx_len, max_chunk_pages=chunk)
@@ -300,10 +300,10 @@ def test_split_and_launch_option_invariance():
                 got = gu.run_verify(q_bits, w.n_q, pool, w.bt_indptr, w.bt_pages, w.ctx_len)
                 _check_pair(got, ref_v, f"verify pdl={pdl} early={early} cluster={cluster}")
     finally:
-        kap.set_launch_options(1, 1, 0, 8, 8)
+        kap.set_launch_options(1, 1, 0, 16, 8)
 
 
-@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+@pytest.mark.parametrize("cluster", [1, 2, 5, 8, 13, 16])
 @pytest.mark.parametrize("cps,ring", [(1, 8), (2, 12), (0, 24), (0, 8)])
 def test_cluster_sizes_on_ragged_batches(cluster, cps, ring):
     """Every cluster size on ragged batches with all row-tile counts (n_q 1..16), including lists
@@ -322,7 +322,7 @@ def test_cluster_sizes_on_ragged_batches(cluster, cps, ring):
                         gu.oracle_verify(q_bits, w.n_q, pool_bits, w.bt_indptr, w.bt_pages, w.ctx_len),
                         f"cluster {cluster} verify {seed}")
     finally:
-        kap.set_launch_options(1, 1, 0, 8, 8)
+        kap.set_launch_options(1, 1, 0, 16, 8)
 
 
 def test_repeated_calls_and_workspace_reuse():
