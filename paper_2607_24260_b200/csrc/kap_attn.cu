@@ -33,7 +33,7 @@ namespace kap {
 
 kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t* n_q,
                           int32_t num_q_heads, int32_t num_kv_heads, const int32_t cluster_slots[kMaxCluster],
-                          int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
+                          const int32_t one_wave_slots[kMaxCluster], int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
                           std::vector<WorkItem>& items, std::vector<MergeGroup>& groups,
                           int32_t* max_chunk_out, int32_t* row_tiles_out, int32_t* cluster_out);
 
@@ -863,8 +863,13 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
         slots[c - 1] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
     }
+    // a one-wave schedule leaves a third of the SM's CTA slots to the next kernel's early CTAs
+    int32_t one_wave[kMaxCluster];
+    const int keep = per_sm >= occ && occ >= 3 ? occ - occ / 3 : per_sm;
+    for (int c = 1; c <= kMaxCluster; ++c)
+        one_wave[c - 1] = (int32_t)((int64_t)slots[c - 1] * keep / per_sm);
     int32_t cluster = 1;
-    kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots,
+    kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots, one_wave,
                                    max_chunk_pages, ws->max_items, ws->max_rows, items, groups,
                                    &max_chunk, &row_tiles, &cluster);
     if (st != KAP_OK) return st;

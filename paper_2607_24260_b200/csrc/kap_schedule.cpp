@@ -9,6 +9,7 @@
 // computed once per request shape and reused for every layer and step.
 #include <algorithm>
 #include <cstring>
+#include <functional>
 #include <numeric>
 #include <vector>
 
@@ -30,14 +31,18 @@ int64_t chunks_for(const int32_t* len, int32_t batch, int32_t hkv, int64_t t) {
 // Cost model used to pick the cluster size and the number of waves, in units of "pages streamed
 // by one CTA": a CTA pays a fixed start-up / epilogue cost, a launch whose groups need more than
 // one cluster pays for the separate merge pass, a cluster pays for its two cluster barriers.
-constexpr int64_t kFixedPages = 6;
+constexpr int64_t kFixedPages = 6;                        // + rows / 2: wider items start and end slower
 constexpr int64_t kMergePassPages = 9;
+constexpr int64_t kLaterWavePages = 40;
 constexpr int64_t kClusterPages = 1;
 constexpr int32_t kDefaultChunkCap = 512;     // per CTA; also the size of the kernel's page-id buffer
 
-// cluster_slots[c - 1] = clusters of c CTAs that can be resident at once (0 = size not allowed)
+// cluster_slots[c - 1] = clusters of c CTAs that can be resident at once (0 = size not allowed);
+// one_wave_slots[c - 1] = how many of them a schedule that fits one wave may use: leaving part of
+// every SM free lets the next kernel's CTAs become resident early (programmatic dependent launch)
 kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t* n_q,
                           int32_t num_q_heads, int32_t num_kv_heads, const int32_t cluster_slots[kMaxCluster],
+                          const int32_t one_wave_slots[kMaxCluster],
                           int32_t max_chunk_pages, int32_t max_items, int32_t max_rows,
                           std::vector<WorkItem>& items, std::vector<MergeGroup>& groups,
                           int32_t* max_chunk_out, int32_t* row_tiles_out, int32_t* cluster_out)
@@ -70,7 +75,16 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
     *cluster_out = 1;
     if (batch == 0) return KAP_OK;
 
-    // smallest cluster-level chunk t with chunks_for(t) <= budget clusters
+    // A candidate schedule = a cluster size C and a number of splits per sequence.  Candidates:
+    // for every allowed C and wave count W, the fewest splits that keep every chunk under the
+    // smallest feasible size for C-slots * W items, then the left-over items handed to the
+    // sequences with the longest chunks (so whole waves are filled); plus "one cluster per
+    // (sequence, KV head)" (no merge pass).  A candidate's cost is the makespan of its items on the
+    // resident cluster slots under longest-first list scheduling - which is what the hardware does
+    // with CTAs handed out in index order - in pages streamed per CTA, plus the fixed costs.
+    const int64_t fixed = kFixedPages + rows / 2;            // start-up + epilogue of one CTA
+    const int64_t n_groups_total = (int64_t)batch * num_kv_heads;
+    const int64_t item_cap = std::max<int64_t>(1, max_items);
     auto min_chunk = [&](int64_t budget) -> int64_t {
         int64_t lo = 1, hi = max_len;
         if (chunks_for(list_len, batch, num_kv_heads, hi) > budget) return -1;
@@ -80,41 +94,84 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
         }
         return lo;
     };
-    int64_t best_t = -1, best_cost = INT64_MAX;
+    std::vector<int32_t> splits(batch), best_splits;
+    std::vector<int64_t> sizes, heap;
+    int64_t best_cost = INT64_MAX;
     int32_t best_c = 1;
-    const int64_t item_cap = std::max<int64_t>(1, max_items);
-    for (int ci = 0; ci < kMaxCluster; ++ci) {
-        const int64_t C = ci + 1;
-        if (cluster_slots[ci] <= 0) continue;
-        auto consider = [&](int64_t t, int64_t waves) {
-            if (t <= 0 || (t + C - 1) / C > cap) return false;
-            const bool merge_pass = t < max_len;            // some group needs more than one cluster
-            const int64_t cost = waves * ((t + C - 1) / C + kFixedPages) + (merge_pass ? kMergePassPages : 0)
-                                 + (C > 1 ? kClusterPages : 0);
-            if (cost < best_cost) { best_cost = cost; best_t = t; best_c = (int32_t)C; }
-            return true;
-        };
-        bool found = false;
-        for (int64_t waves = 1; waves <= 64; ++waves) {
-            const int64_t budget = std::min<int64_t>(item_cap, (int64_t)cluster_slots[ci] * waves);
-            const int64_t t = min_chunk(budget);
-            if (consider(t, waves)) { found = true; if (t <= C) break; }
-            if (budget == item_cap) break;                   // no further items to hand out
+    auto evaluate = [&](int64_t C, int64_t slots) {
+        // per-CTA chunk of each item, longest first
+        sizes.clear();
+        bool merge_pass = false;
+        int64_t total = 0, longest = 0;
+        for (int32_t b = 0; b < batch; ++b) {
+            const int64_t n = splits[b], base = list_len[b] / n, rem = list_len[b] % n;
+            if ((base + (rem ? 1 : 0) + C - 1) / C > cap) return;
+            merge_pass |= n > 1;
+            for (int64_t i = 0; i < n; ++i) {
+                const int64_t sz = (base + (i < rem ? 1 : 0) + C - 1) / C + fixed;
+                for (int32_t g = 0; g < num_kv_heads; ++g) sizes.push_back(sz);
+                total += sz * num_kv_heads;
+                longest = std::max(longest, sz);
+            }
         }
-        if (!found) consider(min_chunk(item_cap), (item_cap + cluster_slots[ci] - 1) / cluster_slots[ci]);
-        // one cluster per (sequence, KV head): slightly longer chunks, but no merge pass
-        const int64_t n_groups = (int64_t)batch * num_kv_heads;
-        if (n_groups <= item_cap)
-            consider(max_len, (n_groups + cluster_slots[ci] - 1) / cluster_slots[ci]);
+        if ((int64_t)sizes.size() > item_cap) return;
+        const int64_t penalty = (merge_pass ? kMergePassPages : 0) + (C > 1 ? kClusterPages : 0);
+        if (std::max(longest, (total + slots - 1) / slots) + penalty >= best_cost) return;   // lower bound
+        int64_t makespan = longest;
+        if ((int64_t)sizes.size() > slots) {
+            std::sort(sizes.begin(), sizes.end(), std::greater<int64_t>());
+            heap.assign((size_t)slots, 0);                   // min-heap of slot finish times
+            auto cmp = std::greater<int64_t>();
+            for (int64_t sz : sizes) {
+                std::pop_heap(heap.begin(), heap.end(), cmp);
+                // a CTA that starts behind another one finds no prefetched pages and cannot hide
+                // its prologue behind the previous kernel: it ramps up from an empty ring
+                heap.back() += sz + (heap.back() > 0 ? kLaterWavePages : 0);
+                makespan = std::max(makespan, heap.back());
+                std::push_heap(heap.begin(), heap.end(), cmp);
+            }
+        }
+        if (makespan + penalty < best_cost) { best_cost = makespan + penalty; best_c = (int32_t)C; best_splits = splits; }
+    };
+    static const int64_t kWaves[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 24, 32, 48, 64, INT32_MAX};
+    for (int ci = 0; ci < kMaxCluster; ++ci) {
+        const int64_t C = ci + 1, slots = cluster_slots[ci];
+        if (slots <= 0) continue;
+        int64_t last_budget = -1;
+        for (int64_t waves : kWaves) {                       // the last entry: as many items as allowed
+            const int64_t budget = std::min<int64_t>(item_cap, waves == 1 ? std::min<int64_t>(slots, one_wave_slots[ci]) : slots * waves);
+            if (budget == last_budget) break;
+            last_budget = budget;
+            const int64_t t = min_chunk(budget);
+            if (t <= 0) continue;
+            int64_t used = 0;
+            for (int32_t b = 0; b < batch; ++b) { splits[b] = (int32_t)((list_len[b] + t - 1) / t); used += (int64_t)splits[b] * num_kv_heads; }
+            // hand the left-over items of the last wave to the sequences with the longest chunks
+            for (int64_t left = budget - used; left >= num_kv_heads; left -= num_kv_heads) {
+                int32_t arg = -1; int64_t worst = 1;
+                for (int32_t b = 0; b < batch; ++b) {
+                    const int64_t chunk = (list_len[b] + splits[b] - 1) / splits[b];
+                    if (chunk > worst) { worst = chunk; arg = b; }
+                }
+                if (arg < 0) break;
+                ++splits[arg];
+            }
+            evaluate(C, slots);
+            if (t <= C) break;                               // chunks cannot get any smaller
+        }
+        if (n_groups_total <= item_cap) {                    // one cluster per (sequence, KV head)
+            std::fill(splits.begin(), splits.end(), 1);
+            evaluate(C, slots);
+        }
     }
-    if (best_t < 0)
+    if (best_cost == INT64_MAX)
         return fail(KAP_ERR_CAPACITY, "page lists need more than %d work items of <= %d pages per CTA",
                     max_items, cap);
 
     int32_t slot = 0;
     for (int32_t b = 0; b < batch; ++b) {
         const int32_t len = list_len[b];
-        const int32_t n_splits = (int32_t)(((int64_t)len + best_t - 1) / best_t);
+        const int32_t n_splits = best_splits[b];
         const int32_t base = len / n_splits, rem = len % n_splits;
         for (int32_t g = 0; g < num_kv_heads; ++g) {
             MergeGroup mg{};
@@ -160,7 +217,7 @@ extern "C" kap_status kap_schedule_host(
     int32_t mc = 0, rt = 1, cl = 1;
     int32_t slots[kap::kMaxCluster];
     for (int i = 0; i < kap::kMaxCluster; ++i) slots[i] = (i + 1) <= std::max(max_cluster, 1) ? cta_slots / (i + 1) : 0;
-    kap_status st = kap::build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots,
+    kap_status st = kap::build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots, slots,
                                         max_chunk_pages, max_items, kap::kRowTile * kap::kMaxRowTiles,
                                         items, groups, &mc, &rt, &cl);
     if (st != KAP_OK) return st;
