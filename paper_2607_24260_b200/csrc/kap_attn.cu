@@ -363,6 +363,22 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             }
         }
     }
+    // Where this lane's two query rows live (row R of the item = query token R / G, head R % G of
+    // the group; null for padding rows), and an L2 prefetch of them: a hint only - L2 is coherent,
+    // the loads themselves come after the wait.
+    const int gid = lane >> 2, tid4 = lane & 3;
+    const uint32_t* q_src[2];
+    int q_tok[2];
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        const int R = rt * kRowTile + gid + half * 8;
+        const bool valid = R < rows;
+        q_tok[half] = valid ? R / p.G : item.n_q - 1;
+        q_src[half] = valid ? reinterpret_cast<const uint32_t*>(
+            p.q + ((q_row0 + q_tok[half]) * p.Hq + item.kv_head * p.G + R % p.G) * kHeadDim) : nullptr;
+        if (valid && tid4 < 2)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(q_src[half] + tid4 * 32) : "memory");
+    }
     // ---- nothing else produced by earlier kernels (Q, fresh KV, partial buffers) is touched above
     pdl_wait();
     KAP_TRACE_POINT(blockIdx.x, 2);
@@ -371,23 +387,16 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     if (!p.early_kv) L = p.ctx_len[item.seq];
     const uint64_t deadline = global_ns() + kWaitBudgetNs;
 
-    const int gid = lane >> 2, tid4 = lane & 3;
     // Q fragments (A operand, 16 rows x 128) straight from global memory, zero for padding rows.
-    // Row R of the item = query token R / G, head R % G of the group.
     uint32_t qf[8][4];
     int pos_row[2];                                          // logical position of rows gid, gid+8
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
-        const int R = rt * kRowTile + gid + half * 8;
-        const bool valid = R < rows;
-        const int j = valid ? R / p.G : item.n_q - 1;
-        pos_row[half] = L - item.n_q + j;
-        const uint32_t* src = reinterpret_cast<const uint32_t*>(
-            p.q + ((q_row0 + j) * p.Hq + item.kv_head * p.G + (valid ? R % p.G : 0)) * kHeadDim);
+        pos_row[half] = L - item.n_q + q_tok[half];
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-            qf[ks][half] = valid ? __ldg(src + ks * 8 + tid4) : 0u;          // cols 16ks + 2tid4
-            qf[ks][half + 2] = valid ? __ldg(src + ks * 8 + 4 + tid4) : 0u;  // cols 16ks + 8 + 2tid4
+            qf[ks][half] = q_src[half] ? __ldg(q_src[half] + ks * 8 + tid4) : 0u;          // cols 16ks + 2tid4
+            qf[ks][half + 2] = q_src[half] ? __ldg(q_src[half] + ks * 8 + 4 + tid4) : 0u;  // cols 16ks + 8 + 2tid4
         }
     }
 
