@@ -215,6 +215,39 @@ kap_status kap_verify_attn(
     kap_workspace* ws, void* cuda_stream);
 
 /*
+ * kap_append_kv - place the K and V rows of newly processed tokens into their physical KV slots
+ * (the paper's slot mapping: Section 3.1 "Selected-KV view materialization"; each proposal step and
+ * the verifier pass write the K/V of the tokens they process, Section 3.2).  Token j of sequence b
+ * goes to logical position ctx_len[b] + j, i.e. page bt_pages[bt_indptr[b] + pos / P], slot
+ * pos % P, for both K and V and every KV head.  With advance != 0 the kernel then sets
+ * ctx_len[b] += n_new[b] on the device, so that a loop "append -> attention" over several decoding
+ * steps can be captured into one CUDA graph.  One CTA per sequence; asynchronous on cuda_stream.
+ *
+ * Running k proposal steps on one compiled plan: compile the plan for the length the sequence
+ * will have at the end of the cycle (ctx_len + k, with the recent window widened by k), and run
+ * the attention calls with the current device ctx_len: pages and slots past ctx_len are masked, so
+ * tokens that have not been appended yet are never seen.
+ *
+ * The block table must already hold a page for every position written.  A position without a
+ * page, a page outside the pool or a negative ctx_len is reported in *device_status
+ * (1 << KAP_ERR_DEVICE_INDEX) and that element is not written.
+ * Errors: KAP_ERR_UNSUPPORTED (shape), KAP_ERR_INVALID_ARG (NULL or misaligned pointer),
+ * KAP_ERR_CUDA.
+ */
+kap_status kap_append_kv(
+    const void* k_new,                 /* DEVICE bf16 [sum n_new, Hkv, d] */
+    const void* v_new,                 /* DEVICE bf16 [sum n_new, Hkv, d] */
+    const int32_t* new_indptr,         /* DEVICE [batch+1], or NULL: one new token per sequence */
+    void* kv_pool, int64_t num_pool_pages,
+    const int32_t* bt_indptr,          /* DEVICE [batch+1] CSR block table */
+    const int32_t* bt_pages,           /* DEVICE */
+    int32_t* ctx_len,                  /* DEVICE [batch], read; updated when advance != 0 */
+    int32_t advance,
+    int32_t batch, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
+    int32_t* device_status,            /* DEVICE int32 or NULL */
+    void* cuda_stream);
+
+/*
  * kap_selected_decode_attn_static - the proposal-path attention of kap_selected_decode_attn for
  * callers that are not allowed to allocate device memory.  (The paper has no counterpart: this is
  * a packaging of the same computation, not another operation.)

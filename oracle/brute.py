@@ -77,3 +77,17 @@ def dense_attention(q_bits, pool_bits, bt_pages, L, visible_pages, n_q, scale=No
             out[j, h] = weights[j, h] @ V[:, h // G, :]
             lse[j, h] = m + np.log(e.sum())
     return out, lse, weights
+
+
+def append_kv(pool_bits, bt_pages, L, k_new_bits, v_new_bits, page_size=16):
+    """Slot mapping written out (Section 3.1, "Selected-KV view materialization": newly scheduled
+    tokens go to their physical KV slots): token j of the n_new new tokens is stored at logical
+    position L + j, i.e. page bt_pages[(L + j) // P], slot (L + j) % P, for K and V and every KV
+    head.  pool_bits [pages, 2, Hkv, P, d] uint16 is modified in place; returns the new length."""
+    n_new = k_new_bits.shape[0]
+    for j in range(n_new):
+        pos = L + j
+        page = int(bt_pages[pos // page_size])
+        pool_bits[page, 0, :, pos % page_size, :] = k_new_bits[j]
+        pool_bits[page, 1, :, pos % page_size, :] = v_new_bits[j]
+    return L + n_new

@@ -623,8 +623,11 @@ kap_attn_merge_kernel(const AttnParams p, const MergeGroup* merge_groups)
 
 // ================================================================================= host side
 namespace {
-
 std::atomic<long long> g_launches{0};
+}
+void count_launch() { g_launches.fetch_add(1); }       // for the library's other translation units
+namespace {
+
 std::atomic<int> g_use_pdl{1};
 std::atomic<int> g_max_cluster{kMaxCluster};       // largest thread-block cluster the scheduler may pick
 std::atomic<int> g_early_kv{1};

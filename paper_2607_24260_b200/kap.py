@@ -39,6 +39,8 @@ SIGNATURES = {
     "kap_selected_decode_attn_static": (C.c_int, [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, C.c_int32,
                                                   C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                   C.c_float, C.c_int32, _vp, _vp, _vp, _vp]),
+    "kap_append_kv": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_int32, C.c_int32,
+                                C.c_int32, C.c_int32, C.c_int32, _vp, _vp]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
     "kap_set_launch_options": (C.c_int, [C.c_int32] * 5),
     "kap_launch_count": (C.c_int64, []),
@@ -242,3 +244,14 @@ def selected_decode_attn_static(q, kv_pool, plan_indptr, plan_phys_pages, plan_l
         _dptr(plan_logical_pages), _dptr(ctx_len), B, Hq, Hkv, d, P, sm_scale, int(num_splits),
         _dptr(out), _dptr(lse), _dptr(device_status), _stream_ptr(stream)))
     return out
+
+
+def append_kv(k_new, v_new, kv_pool, bt_indptr, bt_pages, ctx_len, new_indptr=None, advance=True,
+              device_status=None, stream=None):
+    """kap_append_kv: write the new tokens' K/V rows (bf16 [sum n_new, Hkv, d]) into the paged pool
+    at positions ctx_len[b] .. and, with advance, bump ctx_len on the device."""
+    pages, _, Hkv, P, d = kv_pool.shape
+    _check(lib().kap_append_kv(_dptr(k_new), _dptr(v_new), _dptr(new_indptr), _dptr(kv_pool), int(pages),
+                               _dptr(bt_indptr), _dptr(bt_pages), _dptr(ctx_len), int(bool(advance)),
+                               int(ctx_len.shape[0]), Hkv, d, P, _dptr(device_status),
+                               _stream_ptr(stream)))

@@ -1,0 +1,116 @@
+"""Multi-step proposal loop on the GPU: k steps of "append the new token's K/V -> selected-KV decode
+attention", captured into ONE CUDA graph, on a plan compiled once for the end-of-cycle length.
+Every step's output is compared with the oracle run on a host pool that received the same appends
+(slot mapping stated in oracle/brute.py) with that step's context length."""
+import numpy as np
+import pytest
+import torch
+
+import gpu_util as gu
+from helpers import assert_close
+from oracle import brute
+from oracle import kap_oracle as orc
+from paper_2607_24260_b200 import kap, synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _cycle_case(seed, k_steps, lens):
+    """a batch whose block tables already hold pages for k_steps more tokens"""
+    B = len(lens)
+    w = synth.config2(seed, batch=B, L=max(lens), layers=1)
+    w.ctx_len = np.asarray(lens, dtype=np.int32)
+    end = w.ctx_len + k_steps
+    w.bt_indptr, w.bt_pages, w.num_pool_pages = synth.block_tables(end, "shuffled", seed, "append", spare_pages=3)
+    # spans were drawn for max(lens); clip happens in the compiler
+    return w, end
+
+
+@pytest.mark.parametrize("k_steps,lens", [(4, (1000, 2047, 2048, 333)), (8, (4090, 15, 16)), (6, (777,))])
+def test_append_and_decode_loop_in_one_graph(k_steps, lens):
+    w, end = _cycle_case(3, k_steps, lens)
+    B, Hq, Hkv, d = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim
+    rng = synth.rng_for(3, "append-loop", k_steps)
+    q_bits, pool_bits = synth.host_qkv(w, 3, q_rows=k_steps * B)
+    q_bits = q_bits.reshape(k_steps, B, Hq, d)
+    k_new = synth.normal_bf16((k_steps, B, Hkv, d), 0.5, rng)
+    v_new = synth.normal_bf16((k_steps, B, Hkv, d), 0.5, rng)
+    # plan for the end-of-cycle length: recent window widened by k_steps, budget too
+    plan = kap.compile_plan(end, w.span_indptr, w.span_start, w.span_len, w.span_score,
+                            w.budget_tokens + k_steps, w.n_sink, w.n_recent + k_steps, None, 1.0,
+                            w.bt_indptr, w.bt_pages)
+    pool = gu.bits_to_dev(pool_bits)
+    d_q, d_k, d_v = gu.bits_to_dev(q_bits), gu.bits_to_dev(k_new), gu.bits_to_dev(v_new)
+    d_ctx = gu.i32(w.ctx_len)
+    d_out = torch.zeros_like(d_q)
+    status = torch.zeros(1, dtype=torch.int32, device=gu.DEV)
+    args = (gu.i32(plan["plan_indptr"]), gu.i32(plan["plan_phys_pages"]), gu.i32(plan["plan_logical_pages"]))
+    d_bt_indptr, d_bt_pages = gu.i32(w.bt_indptr), gu.i32(w.bt_pages)
+    ws = kap.Workspace(max_rows_per_item=Hq // Hkv, max_batch=B)
+    ws.schedule(np.diff(plan["plan_indptr"]), None, Hq, Hkv)
+
+    def cycle():
+        for t in range(k_steps):
+            kap.append_kv(d_k[t], d_v[t], pool, d_bt_indptr, d_bt_pages, d_ctx, advance=True, device_status=status)
+            kap.selected_decode_attn(d_q[t], pool, *args, d_ctx, d_out[t], ws)
+
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        cycle()                                   # eager warm-up (also proves the non-graph path)
+    stream.synchronize()
+    eager = gu.dev_bf16_to_f64(d_out)
+    # reset state, capture, replay
+    pool.copy_(gu.bits_to_dev(pool_bits))
+    d_ctx.copy_(gu.i32(w.ctx_len))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        pass
+    with torch.cuda.graph(graph, stream=stream):
+        cycle()
+    pool.copy_(gu.bits_to_dev(pool_bits))
+    d_ctx.copy_(gu.i32(w.ctx_len))
+    d_out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    ws.check()
+    assert int(status.item()) == 0
+    np.testing.assert_array_equal(d_ctx.cpu().numpy(), end)
+    got = gu.dev_bf16_to_f64(d_out)
+    np.testing.assert_array_equal(got, eager)    # graph replay == eager, bit for bit
+
+    # oracle: same appends on the host, plan trimmed to the pages that exist at each step
+    host_pool = pool_bits.copy()
+    L = w.ctx_len.copy()
+    for t in range(k_steps):
+        for b in range(B):
+            bt = w.bt_pages[w.bt_indptr[b]:w.bt_indptr[b + 1]]
+            L[b] = brute.append_kv(host_pool, bt, int(L[b]), k_new[t, b:b + 1], v_new[t, b:b + 1])
+        indptr, phys, logical = [0], [], []
+        for b in range(B):
+            lo, hi = plan["plan_indptr"][b], plan["plan_indptr"][b + 1]
+            keep = plan["plan_logical_pages"][lo:hi].astype(np.int64) * 16 < L[b]
+            phys.append(plan["plan_phys_pages"][lo:hi][keep])
+            logical.append(plan["plan_logical_pages"][lo:hi][keep])
+            indptr.append(indptr[-1] + int(keep.sum()))
+        ref, _, _, _ = orc.selected_decode_attn(q_bits[t], host_pool, indptr, np.concatenate(phys),
+                                                np.concatenate(logical), L)
+        assert_close(got[t], ref, what=f"step {t}")
+        assert gu.normalised_error(got[t], ref) <= 2e-2
+    # the device pool equals the host pool wherever tokens were appended
+    np.testing.assert_array_equal(gu.dev_to_bits(pool), host_pool)
+    ws.close()
+
+
+def test_append_reports_missing_page():
+    w, end = _cycle_case(4, 2, (31,))
+    q_bits, pool_bits = synth.host_qkv(w, 4, q_rows=1)
+    pool = gu.bits_to_dev(pool_bits)
+    knew = gu.bits_to_dev(synth.normal_bf16((1, 8, 128), 0.5, synth.rng_for(4, "x")))
+    status = torch.zeros(1, dtype=torch.int32, device=gu.DEV)
+    short_bt = gu.i32(w.bt_pages[:2])                       # 2 pages = 32 tokens
+    ctx = gu.i32([32])                                      # position 32 needs a third page
+    kap.append_kv(knew, knew, pool, gu.i32([0, 2]), short_bt, ctx, advance=False, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1 << kap.ERR_DEVICE_INDEX
+    np.testing.assert_array_equal(gu.dev_to_bits(pool), pool_bits)     # nothing was written

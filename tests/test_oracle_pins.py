@@ -361,3 +361,30 @@ def test_scale_argument_and_batching():
     one = _decode(c, short)
     np.testing.assert_array_equal(both[0][1], one[0][0])
     np.testing.assert_array_equal(both[0][0], _decode(c, logical)[0][0])
+
+
+def test_append_then_attend_equals_attention_over_the_longer_context():
+    """Slot-mapping pin: appending tokens one by one and decoding after each append equals the
+    dense brute force over a pool that held those tokens from the start."""
+    c = _small_case(12, L=90, n_q=1, spare=4)
+    rng = c["rng"]
+    k_steps = 5
+    n_pages_end = (c["L"] + k_steps + P - 1) // P
+    extra = n_pages_end - c["n_pages"]
+    free = [p for p in range(c["pool"].shape[0]) if p not in set(c["bt"].tolist())]
+    bt = np.concatenate([c["bt"], np.asarray(free[:extra], dtype=np.int32)])
+    k_new = synth.normal_bf16((k_steps, c["Hkv"], c["d"]), 0.5, rng)
+    v_new = synth.normal_bf16((k_steps, c["Hkv"], c["d"]), 0.5, rng)
+    q = synth.normal_bf16((k_steps, c["Hq"], c["d"]), 1.0, rng)
+    final = c["pool"].copy()
+    brute.append_kv(final, bt, c["L"], k_new, v_new)
+    pool, L = c["pool"].copy(), c["L"]
+    for t in range(k_steps):
+        L = brute.append_kv(pool, bt, L, k_new[t:t + 1], v_new[t:t + 1])
+        n_pages = (L + P - 1) // P
+        logical = np.arange(n_pages, dtype=np.int32)
+        out, lse, _, nv = orc.selected_decode_attn(q[t:t + 1], pool, [0, n_pages], bt[logical], logical, [L])
+        b_out, b_lse, _ = brute.dense_attention(q[t:t + 1], final, bt, L, range(n_pages), 1)
+        np.testing.assert_allclose(out, b_out, rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(lse, b_lse, rtol=1e-11)
+        assert np.all(nv == L)
