@@ -248,6 +248,37 @@ kap_status kap_append_kv(
     void* cuda_stream);
 
 /*
+ * kap_top3_accept - the verifier's tolerant acceptance rule (Section 3.2, Eq. 2: the verifier
+ * transition returns the number m of proposed tokens accepted consecutively from the start of the
+ * window and the next carry token; the Top-3 rule accepts a proposed token when it is among the
+ * target model's three best candidates under the full context).
+ *
+ * Sequence b owns logits rows row_indptr[b] .. row_indptr[b+1]-1: its verification window of
+ * k_b + 1 rows (carry row first).  proposed[r] is the token proposed for the position that row r
+ * predicts; the last row of a sequence has no proposal (its entry is ignored).
+ *   top3[r][0..2]  the three highest logits of row r: value descending, lower index first on equal
+ *                  values, NaN ranked below every number (fp32 comparisons on the fp32 inputs:
+ *                  exact, no tolerance).
+ *   accepted[b]    m = the largest m <= k_b with proposed[row i] in top3[row i] for all i < m.
+ *   next_token[b]  top3[row m][0]: the verifier's own best token at the first position that was not
+ *                  accepted, or at the bonus position when all k_b were (the paper leaves the
+ *                  choice of the carry open; this is the reading used here).
+ * logits: DEVICE fp32, row r starts at logits + r * row_stride.  All outputs DEVICE int32; top3 is
+ * [total_rows, 3] and is required (it is also the scratch between the two kernels).
+ * Errors: KAP_ERR_INVALID_ARG (NULL pointer, vocab < 3, row_stride < vocab, negative counts),
+ * KAP_ERR_CUDA.  Asynchronous on cuda_stream.
+ */
+kap_status kap_top3_accept(
+    const float* logits, int64_t row_stride,
+    const int32_t* row_indptr,         /* DEVICE [batch+1] */
+    const int32_t* proposed,           /* DEVICE [total_rows] */
+    int32_t batch, int32_t total_rows, int32_t vocab,
+    int32_t* top3,                     /* DEVICE out [total_rows, 3] */
+    int32_t* accepted,                 /* DEVICE out [batch] */
+    int32_t* next_token,               /* DEVICE out [batch] */
+    void* cuda_stream);
+
+/*
  * kap_selected_decode_attn_static - the proposal-path attention of kap_selected_decode_attn for
  * callers that are not allowed to allocate device memory.  (The paper has no counterpart: this is
  * a packaging of the same computation, not another operation.)

@@ -91,3 +91,29 @@ def append_kv(pool_bits, bt_pages, L, k_new_bits, v_new_bits, page_size=16):
         pool_bits[page, 0, :, pos % page_size, :] = k_new_bits[j]
         pool_bits[page, 1, :, pos % page_size, :] = v_new_bits[j]
     return L + n_new
+
+
+def top3_accept(logits, row_indptr, proposed):
+    """Tolerant acceptance (Section 3.2, Eq. 2 with the Top-3 rule): per row the three best
+    candidates (value descending, lower index first on ties, NaN below everything); m = number of
+    proposed tokens accepted consecutively from the start of each sequence's window; next carry =
+    the best candidate of row m.  logits float32 [rows, V].  Returns (top3, accepted, next)."""
+    x = np.asarray(logits, dtype=np.float32)
+    rows, V = x.shape
+    x = np.where(np.isnan(x), -np.inf, x)
+    top3 = np.zeros((rows, 3), dtype=np.int32)
+    for r in range(rows):
+        order = sorted(range(V), key=lambda i: (-float(x[r, i]), i)) if V <= 64 else \
+            np.lexsort((np.arange(V), -x[r].astype(np.float64)))
+        top3[r] = np.asarray(order[:3], dtype=np.int32)
+    B = len(row_indptr) - 1
+    accepted = np.zeros(B, dtype=np.int32)
+    nxt = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        r0, n = int(row_indptr[b]), int(row_indptr[b + 1] - row_indptr[b])
+        m = 0
+        while m < n - 1 and int(proposed[r0 + m]) in top3[r0 + m].tolist():
+            m += 1
+        accepted[b] = m
+        nxt[b] = top3[r0 + m, 0]
+    return top3, accepted, nxt

@@ -41,6 +41,8 @@ SIGNATURES = {
                                                   C.c_float, C.c_int32, _vp, _vp, _vp, _vp]),
     "kap_append_kv": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_int32, C.c_int32,
                                 C.c_int32, C.c_int32, C.c_int32, _vp, _vp]),
+    "kap_top3_accept": (C.c_int, [_vp, C.c_int64, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
+                                  _vp, _vp]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
     "kap_set_launch_options": (C.c_int, [C.c_int32] * 5),
     "kap_launch_count": (C.c_int64, []),
@@ -255,3 +257,13 @@ def append_kv(k_new, v_new, kv_pool, bt_indptr, bt_pages, ctx_len, new_indptr=No
                                _dptr(bt_indptr), _dptr(bt_pages), _dptr(ctx_len), int(bool(advance)),
                                int(ctx_len.shape[0]), Hkv, d, P, _dptr(device_status),
                                _stream_ptr(stream)))
+
+
+def top3_accept(logits, row_indptr, proposed, top3, accepted, next_token, stream=None):
+    """kap_top3_accept on torch CUDA tensors: logits fp32 [rows, vocab] (row stride taken from the
+    tensor), int32 row_indptr [B+1], proposed [rows]; outputs int32 top3 [rows, 3], accepted [B],
+    next_token [B]."""
+    rows, vocab = logits.shape
+    _check(lib().kap_top3_accept(_dptr(logits), int(logits.stride(0)), _dptr(row_indptr), _dptr(proposed),
+                                 int(row_indptr.shape[0]) - 1, int(rows), int(vocab), _dptr(top3),
+                                 _dptr(accepted), _dptr(next_token), _stream_ptr(stream)))

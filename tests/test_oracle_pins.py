@@ -388,3 +388,39 @@ def test_append_then_attend_equals_attention_over_the_longer_context():
         np.testing.assert_allclose(out, b_out, rtol=1e-11, atol=1e-12)
         np.testing.assert_allclose(lse, b_lse, rtol=1e-11)
         assert np.all(nv == L)
+
+
+# --------------------------------------------------------------------------- Top-3 acceptance
+def test_top3_accept_hand_cases():
+    """Eq. 2 with the Top-3 rule on a window worked by hand (k = 3, vocab 6)."""
+    logits = np.array([
+        [0.1, 2.0, 0.3, 1.5, 1.0, -1.0],     # top3 = 1, 3, 4
+        [5.0, 5.0, 5.0, 5.0, 0.0, 0.0],      # ties: lowest indices first -> 0, 1, 2
+        [0.0, np.nan, 3.0, 1.0, 2.0, np.nan],  # NaN ranks last -> 2, 4, 3
+        [9.0, 0.0, 0.0, 0.0, 0.0, 8.0],      # bonus row -> 0, 5, 1
+    ], dtype=np.float32)
+    cases = [
+        ([4, 2, 3, 0], 3, 0),     # all three accepted (3rd-best, tie-ranked 3rd, 3rd-best) -> bonus row's best
+        ([4, 3, 3, 0], 1, 0),     # second proposal (3) is the 4th of the tie -> m = 1, carry = best of row 1
+        ([0, 0, 2, 0], 0, 1),     # first proposal outside the top 3 -> m = 0, carry = best of row 0
+        ([1, 1, 1, 0], 2, 2),     # NaN-valued token 1 is not a candidate of row 2 -> m = 2, carry = 2
+    ]
+    for proposed, want_m, want_next in cases:
+        top3, m, nxt = brute.top3_accept(logits, [0, 4], proposed)
+        assert top3.tolist() == [[1, 3, 4], [0, 1, 2], [2, 4, 3], [0, 5, 1]]
+        assert (int(m[0]), int(nxt[0])) == (want_m, want_next), proposed
+
+
+def test_top3_matches_argsort_and_prefix_definition():
+    rng = synth.rng_for(0, "top3")
+    x = rng.standard_normal((12, 1000)).astype(np.float32)
+    indptr = [0, 5, 5, 12]                       # one empty window in the middle
+    top3, m, nxt = brute.top3_accept(x, indptr, rng.integers(0, 1000, size=12))
+    np.testing.assert_array_equal(top3, np.argsort(-x, axis=1, kind="stable")[:, :3])
+    # proposing the 2nd-best token everywhere accepts everything; carry = best of the bonus row
+    prop = top3[:, 1].copy()
+    _, m, nxt = brute.top3_accept(x, indptr, prop)
+    assert m.tolist() == [4, 0, 6] and nxt[0] == top3[4, 0] and nxt[2] == top3[11, 0]
+    prop[6] = int(np.argsort(x[6])[0])           # the worst token at the 2nd position of window 3 (rows 5..11)
+    _, m, nxt = brute.top3_accept(x, indptr, prop)
+    assert m.tolist() == [4, 0, 1] and nxt[2] == top3[6, 0]
