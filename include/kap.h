@@ -279,6 +279,27 @@ kap_status kap_top3_accept(
     void* cuda_stream);
 
 /*
+ * kap_phase_model - the paper's cost model of one propose-k / verify cycle and its phase boundary
+ * (Section 4.1 and 4.2, Eqs. 3-15).  HOST only; any consistent unit (bytes, seconds).
+ *   k        proposed tokens per cycle (>= 1)            h  acceptance rate in [0, 1] (Eq. 5)
+ *   s        retained-KV ratio (Eq. 4, >= 0)             kv cost of reading the full KV cache
+ *   w_main   weight cost of one main-model step          w_prop  weight cost of one proposal step
+ *            (self-speculation: w_prop = w_main)
+ * out[8]:  [0] Cost_full = w_main + kv (Eq. 3)           [1] Cost_base = (1 + k h) Cost_full (Eq. 6)
+ *          [2] Cost_plan = k (w_prop + s kv) + Cost_full (Eq. 7)
+ *          [3] speedup = Cost_base / Cost_plan           [4] phase slack = h Cost_full - (w_prop + s kv) (Eq. 13)
+ *          [5] break-even KV: (w_prop - h w_main) / (h - s) when h > s (Eq. 12 in general form; 0 if
+ *              already negative), +inf when h <= s and the right-hand side is positive
+ *          [6] 1 if the plan lies in the positive-speedup region (slack > 0, Eq. 8), else 0
+ *          [7] h - s (Eq. 11)
+ * Cost_base - Cost_plan = k * slack, so k never changes the sign (the paper's first implication).
+ * Errors: KAP_ERR_INVALID_ARG for NULL out, non-finite input, k < 1, h outside [0, 1], negative
+ * s or costs; out is untouched on error.
+ */
+kap_status kap_phase_model(double k, double h, double s, double w_main, double w_prop, double kv,
+                           double* out /* HOST [8] */);
+
+/*
  * kap_selected_decode_attn_static - the proposal-path attention of kap_selected_decode_attn for
  * callers that are not allowed to allocate device memory.  (The paper has no counterpart: this is
  * a packaging of the same computation, not another operation.)

@@ -117,3 +117,21 @@ def top3_accept(logits, row_indptr, proposed):
         accepted[b] = m
         nxt[b] = top3[r0 + m, 0]
     return top3, accepted, nxt
+
+
+def phase_model(k, h, s, w_main, w_prop, kv):
+    """Section 4.1-4.2 written out: Eq. 3 Cost_full, Eq. 6 Cost_base, Eq. 7 Cost_plan, their ratio,
+    Eq. 13 phase slack, the break-even KV scale of Eq. 12 (general form), the Eq. 8 verdict and
+    the Eq. 11 margin.  Plain Python floats (fp64)."""
+    cost_full = w_main + kv
+    cost_base = (1 + k * h) * (w_main + kv)
+    cost_plan = k * (w_prop + s * kv) + (w_main + kv)
+    slack = h * (w_main + kv) - (w_prop + s * kv)
+    rhs = w_prop - h * w_main
+    if h > s:
+        kv_crit = rhs / (h - s) if rhs > 0 else 0.0
+    else:
+        kv_crit = 0.0 if rhs < 0 else float("inf")
+    return dict(cost_full=cost_full, cost_base=cost_base, cost_plan=cost_plan,
+                speedup=cost_base / cost_plan if cost_plan > 0 else float("inf"), slack=slack,
+                kv_crit=kv_crit, beneficial=1.0 if cost_plan < cost_base else 0.0, h_minus_s=h - s)

@@ -43,6 +43,7 @@ SIGNATURES = {
                                 C.c_int32, C.c_int32, C.c_int32, _vp, _vp]),
     "kap_top3_accept": (C.c_int, [_vp, C.c_int64, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
                                   _vp, _vp]),
+    "kap_phase_model": (C.c_int, [C.c_double] * 6 + [C.POINTER(C.c_double)]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
     "kap_set_launch_options": (C.c_int, [C.c_int32] * 5),
     "kap_launch_count": (C.c_int64, []),
@@ -267,3 +268,14 @@ def top3_accept(logits, row_indptr, proposed, top3, accepted, next_token, stream
     _check(lib().kap_top3_accept(_dptr(logits), int(logits.stride(0)), _dptr(row_indptr), _dptr(proposed),
                                  int(row_indptr.shape[0]) - 1, int(rows), int(vocab), _dptr(top3),
                                  _dptr(accepted), _dptr(next_token), _stream_ptr(stream)))
+
+
+PHASE_FIELDS = ("cost_full", "cost_base", "cost_plan", "speedup", "slack", "kv_crit", "beneficial",
+                "h_minus_s")
+
+
+def phase_model(k, h, s, w_main, w_prop, kv):
+    """kap_phase_model: dict of the cost model's quantities (Eqs. 3-15)."""
+    out = (C.c_double * 8)()
+    _check(lib().kap_phase_model(float(k), float(h), float(s), float(w_main), float(w_prop), float(kv), out))
+    return dict(zip(PHASE_FIELDS, [float(x) for x in out]))
