@@ -300,6 +300,30 @@ kap_status kap_phase_model(double k, double h, double s, double w_main, double w
                            double* out /* HOST [8] */);
 
 /*
+ * kap_materialize_view - the paper's selected-KV view as a physical copy (Section 3.1,
+ * "Selected-KV view materialization": the plan's pages are laid out compactly in a reusable
+ * workspace and a compact block table maps the plan's logical blocks to the compact pages).
+ * compact_pool[i] = kv_pool[plan_phys_pages[i]] for i < n_selected, compact_pages[i] = i; logical
+ * page indices are untouched (positions are preserved).  kap_selected_decode_attn run on
+ * (compact_pool, compact_pages, plan_logical_pages) then equals the in-place call bit for bit.
+ * This library's attention gathers in place and does not need the copy; the call is here for
+ * comparison and for back ends that want a dense view.
+ * n_selected > compact_capacity is the paper's "plan exceeds the workspace" fallback condition:
+ * KAP_ERR_CAPACITY, nothing enqueued.  A source page outside the pool is reported in
+ * *device_status (1 << KAP_ERR_DEVICE_INDEX) and not copied.  Other errors: KAP_ERR_UNSUPPORTED
+ * (shape), KAP_ERR_INVALID_ARG, KAP_ERR_CUDA.  Asynchronous on cuda_stream.
+ */
+kap_status kap_materialize_view(
+    const void* kv_pool, int64_t num_pool_pages,   /* DEVICE bf16 [pages][2][Hkv][P][d] */
+    const int32_t* plan_phys_pages,                /* DEVICE [n_selected] */
+    int64_t n_selected,
+    int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
+    void* compact_pool, int64_t compact_capacity,  /* DEVICE bf16 [capacity][2][Hkv][P][d] */
+    int32_t* compact_pages,                        /* DEVICE out [n_selected] or NULL */
+    int32_t* device_status,                        /* DEVICE int32 or NULL */
+    void* cuda_stream);
+
+/*
  * kap_selected_decode_attn_static - the proposal-path attention of kap_selected_decode_attn for
  * callers that are not allowed to allocate device memory.  (The paper has no counterpart: this is
  * a packaging of the same computation, not another operation.)

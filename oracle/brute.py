@@ -135,3 +135,10 @@ def phase_model(k, h, s, w_main, w_prop, kv):
     return dict(cost_full=cost_full, cost_base=cost_base, cost_plan=cost_plan,
                 speedup=cost_base / cost_plan if cost_plan > 0 else float("inf"), slack=slack,
                 kv_crit=kv_crit, beneficial=1.0 if cost_plan < cost_base else 0.0, h_minus_s=h - s)
+
+
+def materialize_view(pool_bits, plan_phys_pages):
+    """The selected-KV view as a copy (Section 3.1, "Selected-KV view materialization"): compact
+    page i holds the plan's i-th page; returns (compact pool, compact page ids)."""
+    phys = np.asarray(plan_phys_pages, dtype=np.int64)
+    return pool_bits[phys].copy(), np.arange(len(phys), dtype=np.int32)

@@ -44,6 +44,8 @@ SIGNATURES = {
     "kap_top3_accept": (C.c_int, [_vp, C.c_int64, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
                                   _vp, _vp]),
     "kap_phase_model": (C.c_int, [C.c_double] * 6 + [C.POINTER(C.c_double)]),
+    "kap_materialize_view": (C.c_int, [_vp, C.c_int64, _vp, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
+                                       _vp, C.c_int64, _vp, _vp, _vp]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
     "kap_set_launch_options": (C.c_int, [C.c_int32] * 5),
     "kap_launch_count": (C.c_int64, []),
@@ -279,3 +281,13 @@ def phase_model(k, h, s, w_main, w_prop, kv):
     out = (C.c_double * 8)()
     _check(lib().kap_phase_model(float(k), float(h), float(s), float(w_main), float(w_prop), float(kv), out))
     return dict(zip(PHASE_FIELDS, [float(x) for x in out]))
+
+
+def materialize_view(kv_pool, plan_phys_pages, compact_pool, compact_pages=None, device_status=None,
+                     stream=None):
+    """kap_materialize_view: copy the plan's pages into compact_pool in plan order."""
+    pages, _, Hkv, P, d = kv_pool.shape
+    _check(lib().kap_materialize_view(_dptr(kv_pool), int(pages), _dptr(plan_phys_pages),
+                                      int(plan_phys_pages.shape[0]), Hkv, d, P, _dptr(compact_pool),
+                                      int(compact_pool.shape[0]), _dptr(compact_pages),
+                                      _dptr(device_status), _stream_ptr(stream)))
