@@ -310,6 +310,82 @@ def time_e2e(cy: Cycle, steps, warmup):
     return (time.perf_counter() - t0) * 1e3 / steps, h2d, d2h
 
 
+# ------------------------------------------------------------------------- the path's other calls
+def time_extras(cy: Cycle, vocab: int = 128256, iters: int = 20):
+    """Side measurements of the calls around the two attention kernels, on the same workload:
+    host plan compilation and scheduling (once per request in the paper), the KV append of one
+    token per sequence, Top-3 acceptance over the verification window's logits, and the compact
+    view copy the paper's design would make once per request.  Not part of `value`."""
+    torch, kap, w = cy.torch, cy.kap, cy.w
+    dev = cy.dev
+    out = {}
+    t0 = time.perf_counter()
+    for _ in range(iters):
+        plan = kap.compile_workload(w)
+    out["compile_plan_ms"] = (time.perf_counter() - t0) / iters * 1e3
+    t0 = time.perf_counter()
+    for _ in range(iters):
+        cy.ws_d.schedule(cy.n_sel, None, w.num_q_heads, w.num_kv_heads, cy.chunks[0])
+    torch.cuda.synchronize()
+    out["schedule_ms"] = (time.perf_counter() - t0) / iters * 1e3
+
+    def timed(fn):
+        """device time per call: `iters` calls captured into one CUDA graph (no host overhead)"""
+        stream = torch.cuda.Stream(device=dev)
+        stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(stream):
+            fn()
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(iters):
+                fn()
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters * 1e3          # us
+
+    # append one token per sequence (positions ctx_len-1 rewritten: ctx is not advanced)
+    k_new = torch.randn((w.batch, w.num_kv_heads, w.head_dim), device=dev).to(torch.bfloat16)
+    ctx_prev = (cy.d_ctx - 1).contiguous()
+    out["append_kv_us"] = timed(lambda: kap.append_kv(k_new, k_new, cy.pool[0], cy.d_bt_indptr, cy.d_bt_pages,
+                                                       ctx_prev, advance=False))
+    # Top-3 acceptance over k + 1 rows per sequence; several logit buffers in turn so that the
+    # rows come from HBM, not from L2
+    rows = w.batch * (cy.k + 1)
+    n_buf = max(2, int(256e6 // (rows * vocab * 4)) + 1)
+    logits = [torch.randn((rows, vocab), device=dev, dtype=torch.float32) for _ in range(n_buf)]
+    indptr = torch.arange(0, rows + 1, cy.k + 1, device=dev, dtype=torch.int32)
+    prop = torch.randint(0, vocab, (rows,), device=dev, dtype=torch.int32)
+    top3 = torch.zeros((rows, 3), device=dev, dtype=torch.int32)
+    acc = torch.zeros(w.batch, device=dev, dtype=torch.int32)
+    nxt = torch.zeros(w.batch, device=dev, dtype=torch.int32)
+    turn = [0]
+
+    def accept():
+        kap.top3_accept(logits[turn[0] % n_buf], indptr, prop, top3, acc, nxt)
+        turn[0] += 1
+    us = timed(accept)
+    out["top3_accept_us"] = us
+    out["top3_accept_GBps"] = rows * vocab * 4 / (us * 1e-6) / 1e9
+    out["top3_accept_shape"] = [rows, vocab]
+    # compact copy of one layer's selected pages (a different layer each call: no L2 reuse)
+    n = int(cy.plan["plan_indptr"][-1])
+    compact = torch.empty((3, n) + tuple(cy.pool.shape[2:]), dtype=torch.bfloat16, device=dev)
+
+    def view():
+        kap.materialize_view(cy.pool[turn[0] % cy.layers], cy.d_plan_phys, compact[turn[0] % 3])
+        turn[0] += 1
+    us = timed(view)
+    out["materialize_view_us_per_layer"] = us
+    out["materialize_view_GBps_read_plus_write"] = 2 * n * w.page_bytes / (us * 1e-6) / 1e9
+    return out
+
+
 # ---------------------------------------------------------------------------------- CPU baseline
 def oracle_cycle_seconds(w, plan, layers_budget_s=12.0, seed=0):
     """Time the oracle, as it stands, on a bounded sample: whole layers of the workload (proposal
@@ -453,6 +529,7 @@ def main():
         e2e_ms = dist.max_float(e2e_ms)
     cy.ws_d.check()
     cy.ws_v.check()
+    extras = time_extras(cy) if (rank == 0 and world == 1) else None
     w, k = cy.w, cy.k
     dominant = "verify" if res["share_decode"] < 0.5 else "decode"
     line = {
@@ -475,6 +552,8 @@ def main():
         "decode_only_tokens_per_s": res["decode_only_tokens_per_s"],
         "retained_kv_ratio_s": res["retained_kv_ratio_s"], "schedule": res["schedule"],
     }
+    if extras:
+        line["other_calls"] = extras
     cy.free()
 
     if rank == 0 and world == 1 and not args.no_sweep and args.config == "c2":

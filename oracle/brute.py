@@ -95,17 +95,18 @@ def append_kv(pool_bits, bt_pages, L, k_new_bits, v_new_bits, page_size=16):
 
 def top3_accept(logits, row_indptr, proposed):
     """Tolerant acceptance (Section 3.2, Eq. 2 with the Top-3 rule): per row the three best
-    candidates (value descending, lower index first on ties, NaN below everything); m = number of
+    candidates (value descending, lower index first on ties, NaN below every number, -inf included); m = number of
     proposed tokens accepted consecutively from the start of each sequence's window; next carry =
     the best candidate of row m.  logits float32 [rows, V].  Returns (top3, accepted, next)."""
     x = np.asarray(logits, dtype=np.float32)
     rows, V = x.shape
-    x = np.where(np.isnan(x), -np.inf, x)
+    nan = np.isnan(x)
+    val = np.where(nan, 0.0, x).astype(np.float64)
     top3 = np.zeros((rows, 3), dtype=np.int32)
     for r in range(rows):
-        order = sorted(range(V), key=lambda i: (-float(x[r, i]), i)) if V <= 64 else \
-            np.lexsort((np.arange(V), -x[r].astype(np.float64)))
-        top3[r] = np.asarray(order[:3], dtype=np.int32)
+        # rank: numbers before NaN, then value descending, then index ascending
+        order = np.lexsort((np.arange(V), -val[r], nan[r]))
+        top3[r] = order[:3]
     B = len(row_indptr) - 1
     accepted = np.zeros(B, dtype=np.int32)
     nxt = np.zeros(B, dtype=np.int32)

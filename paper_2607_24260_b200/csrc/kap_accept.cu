@@ -4,12 +4,13 @@
 // prefix; the next carry token is the verifier's own best candidate at the first position that
 // was not accepted (the bonus position when everything was accepted).
 //
-// Kernel 1: one CTA per logits row finds the row's top 3 (value descending, index ascending on
-// ties, NaN ranked below everything) - a pure streaming reduction over the vocabulary.
+// Kernel 1: a cluster of up to 8 CTAs per logits row finds the row's top 3 (value descending, index ascending on
+// ties, NaN ranked below everything, -inf included) - a pure streaming reduction over the vocabulary.
 // Kernel 2: one thread per sequence walks its rows.
 #include <cuda_runtime.h>
 
 #include <cfloat>
+#include <mutex>
 
 #include "kap_internal.h"
 
@@ -18,68 +19,106 @@ void count_launch();
 
 namespace {
 
-struct Top3 { float v[3]; int i[3]; };
+// A candidate is one 64-bit key that sorts the way the rule ranks: the logit mapped to an
+// order-preserving unsigned integer in the high word (NaN -> 0, below -inf), the complemented index
+// in the low word (lower index wins ties).  Keeping the best three is then five branch-free
+// max / min operations per logit - no divergence, whatever the data.
+typedef unsigned long long Key;
+struct Top3 { Key k[3]; };                                     // k[0] >= k[1] >= k[2]; 0 = empty
 
-// strict "a ranks before b": higher value first, then lower index
-__device__ __forceinline__ bool before(float va, int ia, float vb, int ib) {
-    return va > vb || (va == vb && ia < ib);
+__device__ __forceinline__ Key make_key(float v, int i) {
+    uint32_t u = __float_as_uint(v + 0.0f);                     // -0.0 and +0.0 are the same value
+    u = (v != v) ? 0u : (u ^ ((u >> 31) ? 0xffffffffu : 0x80000000u));
+    return ((Key)u << 32) | (uint32_t)~i;
 }
-__device__ __forceinline__ void push(Top3& t, float v, int i) {
-    if (!(v == v)) v = -INFINITY;                                  // NaN ranks last
-    if (!before(v, i, t.v[2], t.i[2])) return;
-    if (before(v, i, t.v[0], t.i[0])) {
-        t.v[2] = t.v[1]; t.i[2] = t.i[1]; t.v[1] = t.v[0]; t.i[1] = t.i[0]; t.v[0] = v; t.i[0] = i;
-    } else if (before(v, i, t.v[1], t.i[1])) {
-        t.v[2] = t.v[1]; t.i[2] = t.i[1]; t.v[1] = v; t.i[1] = i;
-    } else {
-        t.v[2] = v; t.i[2] = i;
-    }
+__device__ __forceinline__ int key_index(Key k) { return (int)~(uint32_t)k; }
+__device__ __forceinline__ void push(Top3& t, Key x) {
+    const Key b0 = max(t.k[0], x), r1 = min(t.k[0], x);
+    const Key b1 = max(t.k[1], r1), r2 = min(t.k[1], r1);
+    t.k[0] = b0; t.k[1] = b1; t.k[2] = max(t.k[2], r2);
 }
-__device__ __forceinline__ Top3 empty_top3() {
-    Top3 t;
-#pragma unroll
-    for (int k = 0; k < 3; ++k) { t.v[k] = -INFINITY; t.i[k] = INT32_MAX; }
-    return t;
-}
+__device__ __forceinline__ Top3 empty_top3() { Top3 t; t.k[0] = t.k[1] = t.k[2] = 0; return t; }
 
+// grid = rows * S CTAs in clusters of S: the S CTAs of a cluster share one row (a slice of the
+// vocabulary each) and the cluster's first CTA merges their candidates through distributed
+// shared memory.
 __global__ void __launch_bounds__(256)
-kap_top3_rows_kernel(const float* __restrict__ logits, long long row_stride, int vocab,
+kap_top3_rows_kernel(const float* __restrict__ logits, long long row_stride, int vocab, int S,
                      int32_t* __restrict__ top3)
 {
-    const float* row = logits + (long long)blockIdx.x * row_stride;
+    const int r = blockIdx.x / S, part_id = blockIdx.x % S;
+    const float* row = logits + (long long)r * row_stride;
+    const int per = (vocab + S - 1) / S;
+    const int lo = min(vocab, part_id * per), hi = min(vocab, lo + per);
     Top3 t = empty_top3();
-    // 16-byte loads where the row allows it, scalar head and tail otherwise
-    const int head = min(vocab, (int)(((16 - (reinterpret_cast<uintptr_t>(row) & 15)) & 15) / 4));
-    for (int i = threadIdx.x; i < head; i += blockDim.x) push(t, row[i], i);
-    const int n4 = (vocab - head) / 4;
-    const float4* row4 = reinterpret_cast<const float4*>(row + head);
-    for (int j = threadIdx.x; j < n4; j += blockDim.x) {
-        const float4 x = __ldcs(row4 + j);
-        const int i = head + 4 * j;
-        push(t, x.x, i); push(t, x.y, i + 1); push(t, x.z, i + 2); push(t, x.w, i + 3);
+    // 16-byte loads where the slice allows it, scalar head and tail otherwise
+    const int head = min(hi - lo, (int)(((16 - (reinterpret_cast<uintptr_t>(row + lo) & 15)) & 15) / 4));
+    for (int i = lo + threadIdx.x; i < lo + head; i += blockDim.x) push(t, make_key(row[i], i));
+    const int n4 = (hi - lo - head) / 4;
+    const float4* row4 = reinterpret_cast<const float4*>(row + lo + head);
+    for (int j0 = threadIdx.x; j0 < n4; j0 += 8 * blockDim.x) {       // eight loads in flight per thread
+        float4 x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int j = j0 + u * blockDim.x;
+            if (j < n4) x[u] = __ldcs(row4 + j);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int j = j0 + u * blockDim.x;
+            if (j < n4) {
+                const int i = lo + head + 4 * j;
+                push(t, make_key(x[u].x, i)); push(t, make_key(x[u].y, i + 1));
+                push(t, make_key(x[u].z, i + 2)); push(t, make_key(x[u].w, i + 3));
+            }
+        }
     }
-    for (int i = head + 4 * n4 + threadIdx.x; i < vocab; i += blockDim.x) push(t, row[i], i);
+    for (int i = lo + head + 4 * n4 + threadIdx.x; i < hi; i += blockDim.x) push(t, make_key(row[i], i));
     // warp merge, then the 8 warps through shared memory
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
-        Top3 o;
+        Key o[3];
 #pragma unroll
-        for (int k = 0; k < 3; ++k) {
-            o.v[k] = __shfl_xor_sync(0xffffffffu, t.v[k], off);
-            o.i[k] = __shfl_xor_sync(0xffffffffu, t.i[k], off);
-        }
+        for (int k = 0; k < 3; ++k) o[k] = __shfl_xor_sync(0xffffffffu, t.k[k], off);
 #pragma unroll
-        for (int k = 0; k < 3; ++k) push(t, o.v[k], o.i[k]);
+        for (int k = 0; k < 3; ++k) push(t, o[k]);
     }
     __shared__ Top3 part[8];
+    __shared__ Top3 cta_best;
+    __shared__ Top3 peers[8];
     if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = t;
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
 #pragma unroll
-            for (int k = 0; k < 3; ++k) push(t, part[w].v[k], part[w].i[k]);
+            for (int k = 0; k < 3; ++k) push(t, part[w].k[k]);
+        cta_best = t;
+    }
+    if (S > 1) {
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        // thread p of the first CTA fetches peer p's candidates (all peers in parallel), thread 0
+        // merges them
+        if (part_id == 0 && threadIdx.x >= 1 && threadIdx.x < S) {
+            uint32_t addr;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+                         : "=r"(addr) : "r"((uint32_t)__cvta_generic_to_shared(&cta_best)), "r"((int)threadIdx.x));
+            Top3 o;
 #pragma unroll
-        for (int k = 0; k < 3; ++k) top3[(long long)blockIdx.x * 3 + k] = t.i[k];
+            for (int k = 0; k < 3; ++k)
+                asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(o.k[k]) : "r"(addr + 8 * k));
+            peers[threadIdx.x] = o;
+        }
+        __syncthreads();
+        if (part_id == 0 && threadIdx.x == 0)
+            for (int peer = 1; peer < S; ++peer)
+#pragma unroll
+                for (int k = 0; k < 3; ++k) push(t, peers[peer].k[k]);
+        // keep every CTA's shared memory alive until the first CTA has read it
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
+    if (part_id == 0 && threadIdx.x == 0) {
+#pragma unroll
+        for (int k = 0; k < 3; ++k) top3[(long long)r * 3 + k] = key_index(t.k[k]);
     }
 }
 
@@ -118,8 +157,26 @@ extern "C" kap_status kap_top3_accept(
     if (!logits || !row_indptr || !proposed || !top3 || !accepted || !next_token)
         return fail(KAP_ERR_INVALID_ARG, "NULL pointer");
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    kap_top3_rows_kernel<<<(unsigned)total_rows, 256, 0, stream>>>(logits, row_stride, vocab, top3);
-    cudaError_t e = cudaGetLastError();
+    // CTAs per row: about 8K logits each, at most 8 (the portable cluster size; clusters of 16
+    // measured slower here: few of them are resident at a time)
+    int S = 1;
+    while (S < 8 && (int64_t)vocab > (int64_t)S * 8192) S *= 2;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        cudaFuncSetAttribute(kap_top3_rows_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        cudaGetLastError();
+    });
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)total_rows * (unsigned)S);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = S > 1 ? 1 : 0;
+    long long stride = row_stride;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kap_top3_rows_kernel, logits, stride, vocab, S, top3);
     if (e == cudaSuccess) {
         count_launch();
         kap_accept_prefix_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, stream>>>(top3, row_indptr, proposed,

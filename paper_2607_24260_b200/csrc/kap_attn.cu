@@ -186,13 +186,13 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta_
 }
 __device__ __forceinline__ float ld_dsmem_f32(uint32_t addr) {
     float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ float4 ld_dsmem_f32x4(uint32_t addr) {
     float4 v;
     asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
 // Programmatic dependent launch: let the next kernel on the stream start its prologue now ...
@@ -581,9 +581,22 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             Merged res; res.m = -INFINITY; res.l = 0.f; res.o = make_float4(0.f, 0.f, 0.f, 0.f);
             const uint32_t o_addr = smem_u32(all + R * kScratchStride + c4 * 4);
             const uint32_t m_addr = smem_u32(m_flat + R), l_addr = smem_u32(l_flat + R);
-            for (int peer = 0; peer < C; ++peer)
-                merge_into(res, ld_dsmem_f32(map_to_cta(m_addr, peer)), ld_dsmem_f32(map_to_cta(l_addr, peer)),
-                           ld_dsmem_f32x4(map_to_cta(o_addr, peer)));
+            // four peers' states are requested before any of them is used: one round trip through
+            // the cluster's shared-memory network per batch instead of one per peer
+            for (int p0 = 0; p0 < C; p0 += 4) {
+                float pm[4], pl[4];
+                float4 po[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int peer = min(p0 + u, C - 1);
+                    pm[u] = ld_dsmem_f32(map_to_cta(m_addr, peer));
+                    pl[u] = ld_dsmem_f32(map_to_cta(l_addr, peer));
+                    po[u] = ld_dsmem_f32x4(map_to_cta(o_addr, peer));
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (p0 + u < C) merge_into(res, pm[u], pl[u], po[u]);
+            }
             if (single) {
                 store_final(p, q_row0 + R / p.G, item.kv_head * p.G + R % p.G, c4, res);
             } else {

@@ -35,6 +35,8 @@ def test_top3_accept_matches_oracle(V, pad):
         x[2, rng.integers(0, V, size=V // 10)] = np.nan        # NaNs rank last
         x[3, :] = -np.inf                                      # a fully masked row
         x[3, V - 1] = 0.0
+        x[4, :] = np.nan                                        # NaN, -inf and signed zeros together
+        x[4, 5:9] = [-np.inf, -0.0, 0.0, -np.inf]
     ref_top3, _, _ = brute.top3_accept(x, indptr, np.zeros(rows, dtype=np.int32))
     # proposals: mostly inside the top 3, a few outside, so prefixes of every length appear
     proposed = ref_top3[np.arange(rows), rng.integers(0, 3, size=rows)].astype(np.int32)

@@ -405,6 +405,11 @@ def test_top3_accept_hand_cases():
         ([0, 0, 2, 0], 0, 1),     # first proposal outside the top 3 -> m = 0, carry = best of row 0
         ([1, 1, 1, 0], 2, 2),     # NaN-valued token 1 is not a candidate of row 2 -> m = 2, carry = 2
     ]
+    # NaN ranks below -inf, signed zeros tie (lower index first)
+    edge = np.array([[np.nan, -np.inf, -0.0, 0.0, np.nan, -np.inf]], dtype=np.float32)
+    assert brute.top3_accept(edge, [0, 1], [0])[0].tolist() == [[2, 3, 1]]
+    edge2 = np.array([[np.nan, -np.inf, np.nan, np.nan]], dtype=np.float32)
+    assert brute.top3_accept(edge2, [0, 1], [0])[0].tolist() == [[1, 0, 2]]
     for proposed, want_m, want_next in cases:
         top3, m, nxt = brute.top3_accept(logits, [0, 4], proposed)
         assert top3.tolist() == [[1, 3, 4], [0, 1, 2], [2, 4, 3], [0, 5, 1]]
