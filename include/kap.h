@@ -21,7 +21,8 @@
  *   - Plain C, no exceptions, no aborts: every call returns a kap_status; kap_last_error() gives
  *     a thread-local message for the last failure on the calling thread.
  *   - Pointers are marked HOST or DEVICE.  The caller owns every buffer it passes; the library
- *     owns only kap_workspace objects.
+ *     owns only kap_workspace objects.  A workspace belongs to one device and may be used by one
+ *     host thread at a time; different workspaces are independent.
  *   - The attention calls only enqueue kernels on the given CUDA stream and return (asynchronous,
  *     no allocation, no synchronisation; they can be captured into a CUDA graph).  Problems a
  *     kernel detects (a page index outside the pool, a bounded wait that ran out) set a status
@@ -387,11 +388,12 @@ kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);
  *                previous kernel has completed an attention kernel reads only static metadata:
  *                the work list, the page lists and q_indptr.  Those arrays must therefore be
  *                final before the previous kernel was launched.
- *   early_kv     != 0 (default; needs use_pdl): in that window the kernel also reads ctx_len and
- *                starts loading KV pages that hold only tokens older than the query rows' own
- *                (t < ctx_len - n_q) - pages written in earlier decoding steps.  ctx_len and those
- *                pages must then be final before the previous kernel was launched; Q, the pages
- *                holding the rows' own tokens, out and lse may still be written by it.
+ *   early_kv     != 0 (default; needs use_pdl): in that window the kernel also reads ctx_len as a
+ *                hint and starts loading KV pages that hold only tokens older than the query
+ *                rows' own (t < ctx_len - n_q) - pages written in earlier decoding steps.  Those
+ *                pages must then be final before the previous kernel was launched, and ctx_len may
+ *                only grow while it runs (the masks use the value read after the wait); Q, the
+ *                pages holding the rows' own tokens, out and lse may still be written by it.
  *   ctas_per_sm  resident CTAs per SM the scheduler fills in one wave; 0 = as many as fit.
  *   max_cluster  largest thread-block cluster (1 .. 16; default 16, sizes above 8 use the
  *                non-portable cluster launch) the scheduler may give a work item.  The CTAs of a cluster share the item's pages and reduce their partial

@@ -349,12 +349,14 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     // Early KV prefetch: pages that hold only tokens older than the query rows' own tokens
     // (t < L - n_q) were written in earlier steps, so their loads may start before the previous
     // kernel on the stream has completed.  Pages holding the rows' own tokens, Q and the partial
-    // buffers wait for it.  (ctx_len must then be final before the previous kernel was launched.)
-    int filled = 0, L = 0;
+    // buffers wait for it.  (ctx_len may only grow while the previous kernel runs.)
+    int filled = 0;
     if (p.early_kv) {
-        L = p.ctx_len[item.seq];
+        // a hint only: if the previous kernel is still advancing ctx_len, an older (smaller) value
+        // just makes fewer pages eligible; the masks use the value read after the wait
+        const int L_hint = p.ctx_len[item.seq];
         if (producer) {
-            const int fresh_from = L - item.n_q;
+            const int fresh_from = L_hint - item.n_q;
             while (filled < depth) {
                 const int idx = first_idx + filled * idx_stride;
                 if (idx >= n_pages || tail->logical[idx] * kPageSize + kPageSize - 1 >= fresh_from) break;
@@ -384,7 +386,7 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     KAP_TRACE_POINT(blockIdx.x, 2);
     if (producer)
         for (; filled < depth; ++filled) fill(grp * depth + filled, filled);
-    if (!p.early_kv) L = p.ctx_len[item.seq];
+    const int L = p.ctx_len[item.seq];
     const uint64_t deadline = global_ns() + kWaitBudgetNs;
 
     // Q fragments (A operand, 16 rows x 128) straight from global memory, zero for padding rows.
@@ -708,24 +710,21 @@ unsigned long long* g_trace = nullptr;      // [g_trace_cap launches][8192][8]
 int g_trace_cap = 0, g_trace_next = 0;
 #endif
 
-std::once_flag g_attr_once;
-cudaError_t g_attr_err = cudaSuccess;
-
 kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pages,
                             kap_workspace* ws, cudaStream_t stream) {
     if (ws->n_items == 0) return KAP_OK;
     const CUtensorMap* map = nullptr;
     kap_status st = get_tensor_map(ws, pool, pages, p_in.Hkv, &map);
     if (st != KAP_OK) return st;
-    std::call_once(g_attr_once, [] {
-        g_attr_err = cudaFuncSetAttribute(kap_attn_split_kernel,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          smem_bytes_for(kMaxSlots));
+    // function attributes are per device: set them once for the workspace's device
+    if (!ws->attrs_set) {
+        cudaError_t ae = cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              smem_bytes_for(kMaxSlots));
+        if (ae != cudaSuccess) return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ae));
         cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         cudaGetLastError();
-    });
-    if (g_attr_err != cudaSuccess)
-        return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(g_attr_err));
+        ws->attrs_set = 1;
+    }
 
     AttnParams p = p_in;
     p.cluster = ws->cluster_size;

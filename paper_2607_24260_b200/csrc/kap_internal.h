@@ -44,7 +44,7 @@ struct MergeGroup {
 struct kap_workspace {
     int32_t device = 0;
     int32_t max_items = 0, max_rows = 0, max_batch = 0;
-    int32_t sm_count = 0, occupancy = 1;
+    int32_t sm_count = 0, occupancy = 1, attrs_set = 0;
     int32_t cluster_size = 1, max_nq = 1, ring_slots = 8;   // of the last schedule
     // last schedule
     int32_t batch = 0, n_items = 0, n_groups = 0, n_merge_groups = 0, max_chunk = 0;
