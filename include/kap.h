@@ -125,7 +125,8 @@ kap_status kap_compile_plan(
  * near-equal contiguous chunks so that the chunks fill the GPU in whole waves, uploads the work
  * list on `cuda_stream` (asynchronous copy from pinned memory owned by the workspace) and keeps
  * it until the next kap_schedule.  The schedule depends only on the page counts, so one schedule
- * serves every layer and every step whose list lengths and row counts are unchanged.
+ * serves every layer and every step whose list lengths and row counts are unchanged; a call that
+ * repeats the previous call's counts and options returns at once and uploads nothing.
  * A workspace serves one attention call at a time: use one for the proposal path and another for
  * the verification path.  max_chunk_pages = 0 picks the default chunk cap.
  * Errors: KAP_ERR_INVALID_ARG (NULL, batch < 0 or > max_batch, list_len <= 0, n_q < 1, bad head

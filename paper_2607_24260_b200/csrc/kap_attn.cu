@@ -844,6 +844,7 @@ extern "C" void kap_workspace_destroy(kap_workspace* ws) {
     cudaFreeHost(ws->h_status);
     if (ws->upload_event) cudaEventDestroy((cudaEvent_t)ws->upload_event);
     delete[] ws->maps;
+    delete ws->schedule_key;
     delete ws;
 }
 
@@ -852,6 +853,15 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
                                    int32_t max_chunk_pages, void* cuda_stream) {
     if (!ws) return fail(KAP_ERR_INVALID_ARG, "NULL workspace");
     if (batch > ws->max_batch) return fail(KAP_ERR_CAPACITY, "batch %d > workspace max_batch %d", batch, ws->max_batch);
+    // The schedule depends only on these numbers: when they repeat (every decoding step of an
+    // unchanged batch), the work list already on the device is the answer.
+    std::vector<int32_t> key;
+    key.reserve(2 * (size_t)std::max(batch, 0) + 8);
+    key.push_back(batch); key.push_back(num_q_heads); key.push_back(num_kv_heads);
+    key.push_back(max_chunk_pages); key.push_back(n_q != nullptr);
+    key.push_back(g_ring_slots.load()); key.push_back(g_ctas_per_sm.load()); key.push_back(g_max_cluster.load());
+    for (int32_t b = 0; b < batch && list_len; ++b) { key.push_back(list_len[b]); key.push_back(n_q ? n_q[b] : 1); }
+    if (ws->schedule_key && *ws->schedule_key == key) return KAP_OK;
     std::vector<WorkItem> items;
     std::vector<MergeGroup> groups;
     int32_t max_chunk = 0, row_tiles = 1;
@@ -928,6 +938,8 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     int32_t mq = 1;
     for (int32_t b = 0; b < batch; ++b) mq = std::max(mq, n_q ? n_q[b] : 1);
     ws->max_nq = mq;
+    if (!ws->schedule_key) ws->schedule_key = new std::vector<int32_t>();
+    *ws->schedule_key = std::move(key);
     return KAP_OK;
 }
 

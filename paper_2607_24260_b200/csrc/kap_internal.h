@@ -3,6 +3,7 @@
 #include <cstdarg>
 #include <cstdint>
 #include <cstdio>
+#include <vector>
 
 #include "kap.h"
 
@@ -70,4 +71,5 @@ struct kap_workspace {
     static constexpr int kMapSlots = 64;
     MapSlot* maps = nullptr;
     int32_t map_next = 0, map_count = 0;
+    std::vector<int32_t>* schedule_key = nullptr;   // inputs of the schedule held on the device
 };
