@@ -39,3 +39,39 @@ def test_no_oracle_import_in_product_path():
                 assert "oracle" not in src.replace("kap_oracle", "oracle") or f == "synth.py" or \
                     "import oracle" not in src and "from oracle" not in src
                 assert "import oracle" not in src and "from oracle" not in src
+
+
+def test_header_is_plain_c_and_links_from_c(tmp_path):
+    """include/kap.h compiles as C99 on its own, and a C program linked against the library can call
+    a host entry point (kap_compile_plan on the hand-worked example) - no C++ or torch types cross
+    the boundary."""
+    import subprocess
+    src = tmp_path / "use_kap.c"
+    src.write_text(r'''
+#include "kap.h"
+#include <stdio.h>
+int main(void) {
+    int32_t ctx[1] = {100}, indptr[2] = {0, 6};
+    int32_t start[6] = {20, 25, 60, 40, 90, 70}, len[6] = {10, 20, 12, 30, 20, 5};
+    float score[6] = {0.9f, 0.8f, 0.8f, 0.5f, 0.95f, 0.4f};
+    int32_t budget[1] = {48}, sink[1] = {4}, recent[1] = {8};
+    int32_t bt_indptr[2] = {0, 7}, bt[7] = {17, 3, 9, 12, 5, 30, 2};
+    int32_t out_indptr[2], logical[7], phys[7], flags[1], sel[1];
+    kap_status st = kap_compile_plan(1, 16, ctx, indptr, start, len, score, budget, sink, recent, 0, 1.0f,
+                                     bt_indptr, bt, 7, out_indptr, logical, phys, flags, sel);
+    if (st != KAP_OK) { printf("error %d: %s\n", (int)st, kap_last_error()); return 1; }
+    printf("%s |", kap_version());
+    for (int i = 0; i < out_indptr[1]; ++i) printf(" %d:%d", logical[i], phys[i]);
+    printf(" | %d %d\n", sel[0], flags[0]);
+    return 0;
+}
+''')
+    inc = os.path.join(ROOT, "include")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-x", "c",
+                    os.path.join(inc, "kap.h")], check=True)
+    lib = build.build()
+    exe = tmp_path / "use_kap"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", inc, str(src), "-o", str(exe), lib,
+                    "-Wl,-rpath," + os.path.dirname(lib)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout
+    assert out.strip().endswith("| 0:17 1:3 2:9 4:5 5:30 6:2 | 44 0"), out
