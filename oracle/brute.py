@@ -43,10 +43,12 @@ def plan_pages(L, spans, budget, n_sink, n_recent, page_size=16, force_full=Fals
     return sorted({t // page_size for t in tokens}), len(tokens), over
 
 
-def dense_attention(q_bits, pool_bits, bt_pages, L, visible_pages, n_q, scale=None):
+def dense_attention(q_bits, pool_bits, bt_pages, L, visible_pages, n_q, scale=None,
+                    visible_tokens=None):
     """One sequence.  q_bits [n_q, Hq, d]; pool_bits [pages, 2, Hkv, P, d]; bt_pages: the
     sequence's block table (logical -> physical); visible_pages: iterable of logical pages the
-    rows may see (all pages for verification).  Row j sits at position L - n_q + j.
+    rows may see (all pages for verification); visible_tokens, when given, replaces it by an
+    explicit set of token positions.  Row j sits at position L - n_q + j.
     Returns (out [n_q, Hq, d], lse [n_q, Hq], weights [n_q, Hq, L])."""
     q = _bf16_to_f64(q_bits)
     pool = _bf16_to_f64(pool_bits)
@@ -62,6 +64,9 @@ def dense_attention(q_bits, pool_bits, bt_pages, L, visible_pages, n_q, scale=No
     page_vis = np.zeros(n_pages, dtype=bool)
     page_vis[list(visible_pages)] = True
     tok_vis = np.repeat(page_vis, P)[:L]
+    if visible_tokens is not None:
+        tok_vis = np.zeros(L, dtype=bool)
+        tok_vis[sorted(visible_tokens)] = True
     out = np.zeros((n_q, Hq, d))
     lse = np.zeros((n_q, Hq))
     weights = np.zeros((n_q, Hq, L))

@@ -72,9 +72,10 @@ int kap_oracle_compile_plan(
     const int32_t* n_recent, const uint8_t* force_full, float s_max,
     const int32_t* bt_indptr, const int32_t* bt_pages, int64_t plan_capacity,
     int32_t* plan_indptr, int32_t* plan_logical_pages, int32_t* plan_phys_pages,
-    int32_t* plan_flags, int32_t* selected_tokens)
+    int32_t* plan_flags, int32_t* selected_tokens, uint16_t* plan_token_masks)
 {
     if (batch < 0 || page_size <= 0) return ORC_INVALID;
+    if (plan_token_masks && page_size > 16) return ORC_INVALID;   /* one bit per token of a page */
     /* validate everything first so that outputs stay untouched on error */
     for (int32_t b = 0; b < batch; ++b) {
         if (ctx_len[b] <= 0 || budget_tokens[b] < 0 || n_sink[b] < 0 || n_recent[b] < 0)
@@ -94,6 +95,7 @@ int kap_oracle_compile_plan(
     int32_t* flags_tmp = (int32_t*)malloc(sizeof(int32_t) * (size_t)(batch + 1));
     int32_t* used_tmp = (int32_t*)malloc(sizeof(int32_t) * (size_t)(batch + 1));
     uint8_t** page_sel = (uint8_t**)calloc((size_t)batch + 1, sizeof(uint8_t*));
+    uint8_t** tok_sel = (uint8_t**)calloc((size_t)batch + 1, sizeof(uint8_t*));
     indptr_tmp[0] = 0;
     int rc = ORC_OK;
 
@@ -160,7 +162,7 @@ int kap_oracle_compile_plan(
         indptr_tmp[b + 1] = (int32_t)written;
         flags_tmp[b] = flags;
         used_tmp[b] = used;
-        free(tok);
+        tok_sel[b] = tok;
     }
     if (written > plan_capacity) rc = ORC_CAPACITY;
     if (rc == ORC_OK) {
@@ -171,6 +173,12 @@ int kap_oracle_compile_plan(
                 if (!page_sel[b][p]) continue;
                 plan_logical_pages[o] = p;
                 if (plan_phys_pages && bt_indptr) plan_phys_pages[o] = bt_pages[bt_indptr[b] + p];
+                if (plan_token_masks) {                       /* bit t: token p*P + t is selected */
+                    uint16_t m = 0;
+                    for (int32_t t = 0; t < page_size && p * page_size + t < ctx_len[b]; ++t)
+                        if (tok_sel[b][p * page_size + t]) m |= (uint16_t)(1u << t);
+                    plan_token_masks[o] = m;
+                }
                 ++o;
             }
             plan_flags[b] = flags_tmp[b];
@@ -178,8 +186,8 @@ int kap_oracle_compile_plan(
         }
         memcpy(plan_indptr, indptr_tmp, sizeof(int32_t) * (size_t)(batch + 1));
     }
-    for (int32_t b = 0; b < batch; ++b) free(page_sel[b]);
-    free(page_sel); free(indptr_tmp); free(flags_tmp); free(used_tmp);
+    for (int32_t b = 0; b < batch; ++b) { free(page_sel[b]); free(tok_sel[b]); }
+    free(page_sel); free(tok_sel); free(indptr_tmp); free(flags_tmp); free(used_tmp);
     return rc;
 }
 
@@ -190,7 +198,8 @@ int kap_oracle_compile_plan(
  * visible tokens; out[d], *lse and *wsum (sum of the normalised weights) are written. */
 static int64_t attend_row(
     const double* q, const uint16_t* pool, int32_t n_list, const int32_t* list_phys,
-    const int32_t* list_logical, int32_t pos, int32_t kv_head, int32_t Hkv, int32_t d, int32_t P,
+    const int32_t* list_logical, const uint16_t* list_masks, int32_t pos, int32_t kv_head, int32_t Hkv,
+    int32_t d, int32_t P,
     double scale, double* logits, double* out, double* lse, double* wsum)
 {
     const int64_t page_stride = (int64_t)2 * Hkv * P * d;
@@ -204,6 +213,7 @@ static int64_t attend_row(
         for (int32_t s = 0; s < P; ++s) {
             const int64_t t = (int64_t)logical * P + s;
             if (t > pos) continue;
+            if (list_masks && !((list_masks[i] >> s) & 1)) continue;   /* token-granular visibility */
             double dot = 0.0;
             for (int32_t c = 0; c < d; ++c) dot += q[c] * bf16_to_double(kpage[(int64_t)s * d + c]);
             const double z = scale * dot;
@@ -222,6 +232,7 @@ static int64_t attend_row(
         for (int32_t s = 0; s < P; ++s) {
             const int64_t t = (int64_t)logical * P + s;
             if (t > pos) continue;
+            if (list_masks && !((list_masks[i] >> s) & 1)) continue;
             const double w = exp(logits[k++] - zmax);
             denom += w;
             for (int32_t c = 0; c < d; ++c) out[c] += w * bf16_to_double(vpage[(int64_t)s * d + c]);
@@ -244,7 +255,7 @@ static int64_t attend_row(
 static int attention(
     const uint16_t* q, const int32_t* q_indptr, const uint16_t* pool, int64_t num_pool_pages,
     const int32_t* list_indptr, const int32_t* list_phys, const int32_t* list_logical,
-    const int32_t* ctx_len, int32_t batch, int32_t Hq, int32_t Hkv, int32_t d, int32_t P,
+    const uint16_t* list_masks, const int32_t* ctx_len, int32_t batch, int32_t Hq, int32_t Hkv, int32_t d, int32_t P,
     double scale, double* out, double* lse, double* wsum, int64_t* n_visible)
 {
     if (batch < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv || d <= 0 || P <= 0) return ORC_INVALID;
@@ -278,7 +289,8 @@ static int attention(
                     qd[c] = bf16_to_double(q[(row * Hq + h) * d + c]);
                 double w = 0.0, l = 0.0;
                 int64_t nv = attend_row(qd, pool, n_list, list_phys + list_indptr[b],
-                                        list_logical ? list_logical + list_indptr[b] : NULL, pos,
+                                        list_logical ? list_logical + list_indptr[b] : NULL,
+                                        list_masks ? list_masks + list_indptr[b] : NULL, pos,
                                         h / G, Hkv, d, P, scale, logits,
                                         out + (row * Hq + h) * d, &l, &w);
                 if (lse) lse[row * Hq + h] = l;
@@ -295,12 +307,14 @@ static int attention(
 int kap_oracle_selected_decode_attn(
     const uint16_t* q, const uint16_t* pool, int64_t num_pool_pages,
     const int32_t* plan_indptr, const int32_t* plan_phys_pages, const int32_t* plan_logical_pages,
-    const int32_t* ctx_len, int32_t batch, int32_t Hq, int32_t Hkv, int32_t d, int32_t P,
+    const uint16_t* plan_token_masks, const int32_t* ctx_len, int32_t batch, int32_t Hq,
+    int32_t Hkv, int32_t d, int32_t P,
     double scale, double* out, double* lse, double* wsum, int64_t* n_visible)
 {
+    if (plan_token_masks && P > 16) return ORC_INVALID;
     return attention(q, NULL, pool, num_pool_pages, plan_indptr, plan_phys_pages,
-                     plan_logical_pages, ctx_len, batch, Hq, Hkv, d, P, scale, out, lse, wsum,
-                     n_visible);
+                     plan_logical_pages, plan_token_masks, ctx_len, batch, Hq, Hkv, d, P, scale,
+                     out, lse, wsum, n_visible);
 }
 
 /* Section 3.2, "Full-context verification": q is [sum n_q, Hq, d]; the page list is the whole
@@ -329,7 +343,7 @@ int kap_oracle_verify_attn(
         memcpy(pages + indptr[b], bt_pages + bt_indptr[b], sizeof(int32_t) * (size_t)n_pages);
         indptr[b + 1] = indptr[b] + n_pages;
     }
-    int rc = attention(q, q_indptr, pool, num_pool_pages, indptr, pages, NULL, ctx_len, batch, Hq,
+    int rc = attention(q, q_indptr, pool, num_pool_pages, indptr, pages, NULL, NULL, ctx_len, batch, Hq,
                        Hkv, d, P, scale, out, lse, wsum, n_visible);
     free(indptr); free(pages);
     return rc;

@@ -43,7 +43,8 @@ def compile_plan(ctx_len, span_indptr, span_start, span_len, span_score, budget_
                  page_size=16, capacity=None):
     """Algorithm 1 (budgeted span selection -> page list).  Returns a dict with plan_indptr,
     plan_logical_pages, plan_phys_pages (None without a block table), plan_flags,
-    selected_tokens."""
+    selected_tokens, plan_token_masks (uint16 per listed page: bit t set when token
+    page*page_size + t is in the selected union U; page_size <= 16 only, else None)."""
     ctx_len = _arr(ctx_len, np.int32)
     B = ctx_len.shape[0]
     span_indptr = _arr(span_indptr, np.int32)
@@ -63,19 +64,22 @@ def compile_plan(ctx_len, span_indptr, span_start, span_len, span_score, budget_
     phys = np.full(max(1, capacity), -1, dtype=np.int32) if bt_indptr is not None else None
     flags = np.full(B, -1, dtype=np.int32)
     sel = np.full(B, -1, dtype=np.int32)
+    masks = np.zeros(max(1, capacity), dtype=np.uint16) if page_size <= 16 else None
     rc = lib().kap_oracle_compile_plan(
         C.c_int32(B), C.c_int32(page_size), _p(ctx_len, C.c_int32), _p(span_indptr, C.c_int32),
         _p(span_start, C.c_int32), _p(span_len, C.c_int32), _p(span_score, C.c_float),
         _p(budget_tokens, C.c_int32), _p(n_sink, C.c_int32), _p(n_recent, C.c_int32),
         _p(force_full, C.c_uint8), C.c_float(s_max), _p(bt_indptr, C.c_int32),
         _p(bt_pages, C.c_int32), C.c_int64(capacity), _p(indptr, C.c_int32),
-        _p(logical, C.c_int32), _p(phys, C.c_int32), _p(flags, C.c_int32), _p(sel, C.c_int32))
+        _p(logical, C.c_int32), _p(phys, C.c_int32), _p(flags, C.c_int32), _p(sel, C.c_int32),
+        _p(masks, C.c_uint16))
     if rc != OK:
         raise OracleError(rc)
     n = int(indptr[-1])
     return dict(plan_indptr=indptr, plan_logical_pages=logical[:n].copy(),
                 plan_phys_pages=None if phys is None else phys[:n].copy(), plan_flags=flags,
-                selected_tokens=sel)
+                selected_tokens=sel,
+                plan_token_masks=None if masks is None else masks[:n].copy())
 
 
 def compile_workload(w, capacity=None):
@@ -90,8 +94,9 @@ def _attn_out(rows, Hq, d):
 
 
 def selected_decode_attn(q_bits, pool_bits, plan_indptr, plan_phys_pages, plan_logical_pages,
-                         ctx_len, scale=None):
-    """q_bits [B, Hq, d] uint16, pool_bits [pages, 2, Hkv, P, d] uint16.
+                         ctx_len, scale=None, plan_token_masks=None):
+    """q_bits [B, Hq, d] uint16, pool_bits [pages, 2, Hkv, P, d] uint16.  plan_token_masks
+    (uint16 per listed page) narrows visibility from whole pages to the tokens whose bit is set.
     Returns (out f64 [B,Hq,d], lse f64 [B,Hq], weight_sum [B,Hq], n_visible [B,Hq])."""
     q_bits = _arr(q_bits, np.uint16)
     pool_bits = _arr(pool_bits, np.uint16)
@@ -102,9 +107,11 @@ def selected_decode_attn(q_bits, pool_bits, plan_indptr, plan_phys_pages, plan_l
     out, lse, ws, nv = _attn_out(B, Hq, d)
     pi, pp = _arr(plan_indptr, np.int32), _arr(plan_phys_pages, np.int32)
     pl, cl = _arr(plan_logical_pages, np.int32), _arr(ctx_len, np.int32)
+    pm = _arr(plan_token_masks, np.uint16)
     rc = lib().kap_oracle_selected_decode_attn(
         _p(q_bits, C.c_uint16), _p(pool_bits, C.c_uint16), C.c_int64(n_pages),
-        _p(pi, C.c_int32), _p(pp, C.c_int32), _p(pl, C.c_int32), _p(cl, C.c_int32),
+        _p(pi, C.c_int32), _p(pp, C.c_int32), _p(pl, C.c_int32), _p(pm, C.c_uint16),
+        _p(cl, C.c_int32),
         C.c_int32(B), C.c_int32(Hq), C.c_int32(Hkv), C.c_int32(d), C.c_int32(P),
         C.c_double(scale), _p(out, C.c_double), _p(lse, C.c_double), _p(ws, C.c_double),
         _p(nv, C.c_int64))

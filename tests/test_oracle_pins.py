@@ -127,6 +127,15 @@ def test_plan_invariants_and_bruteforce_random():
             phys = r["plan_phys_pages"][r["plan_indptr"][b]:r["plan_indptr"][b + 1]]
             bt = w.bt_pages[w.bt_indptr[b]:w.bt_indptr[b + 1]]
             assert phys.tolist() == bt[got].tolist()
+            # token masks: bit t of page p <=> token p*P + t is in the brute-force union U
+            tokens = (set(range(L)) if w.force_full[b] else
+                      brute.plan_tokens(L, spans, int(w.budget_tokens[b]), int(w.n_sink[b]),
+                                        int(w.n_recent[b]))[0])
+            masks = r["plan_token_masks"][r["plan_indptr"][b]:r["plan_indptr"][b + 1]]
+            from_masks = {int(pg) * w.page_size + t for pg, m in zip(got, masks)
+                          for t in range(w.page_size) if (int(m) >> t) & 1}
+            assert from_masks == tokens, (seed, b)
+            assert np.all(masks != 0)
             n_seq += 1
     assert n_seq >= 10_000
 
@@ -157,11 +166,12 @@ def _small_case(seed, L=150, n_q=3, Hq=8, Hkv=2, d=32, spare=5, q_std=1.0, kv_st
                 rng=rng)
 
 
-def _decode(c, logical, q=None, pool=None, L=None):
+def _decode(c, logical, q=None, pool=None, L=None, masks=None):
     logical = np.asarray(logical, dtype=np.int32)
     q = c["q"][-1:] if q is None else q
     return orc.selected_decode_attn(q, c["pool"] if pool is None else pool, [0, len(logical)],
-                                    c["bt"][logical], logical, [c["L"] if L is None else L])
+                                    c["bt"][logical], logical, [c["L"] if L is None else L],
+                                    plan_token_masks=masks)
 
 
 def _verify(c, q=None, pool=None):
@@ -214,6 +224,77 @@ def test_selected_view_equals_masked_full_attention(seed):
     np.testing.assert_allclose(v_lse, b_lse, rtol=1e-11)
     for j in range(c["n_q"]):
         assert np.all(v_nv[j] == c["L"] - c["n_q"] + j + 1)
+
+
+def _random_token_masks(c, logical, rng, density=0.5):
+    """Per listed page a random non-empty 16-bit mask; returns (masks, set of visible tokens)."""
+    masks = np.zeros(len(logical), dtype=np.uint16)
+    tokens = set()
+    for i, lp in enumerate(logical):
+        bits = rng.random(P) < density
+        bits[int(rng.integers(0, min(P, c["L"] - lp * P)))] = True
+        masks[i] = sum(1 << t for t in range(P) if bits[t])
+        tokens |= {int(lp) * P + t for t in range(P) if bits[t] and lp * P + t < c["L"]}
+    return masks, tokens
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_token_masked_view_equals_dense_attention_over_the_token_set(seed):
+    """Token-granular visibility: the masked page-list attention equals dense attention in which
+    exactly the tokens whose bit is set may be seen (numpy brute force over token positions);
+    bits beyond the context end are ignored; an all-ones mask changes nothing."""
+    c = _small_case(40 + seed, L=int(synth.rng_for(seed, "Lm").integers(20, 260)))
+    rng = c["rng"]
+    keep = rng.random(c["n_pages"]) < 0.5
+    keep[-1] = True
+    logical = np.nonzero(keep)[0]
+    masks, tokens = _random_token_masks(c, logical, rng)
+    out, lse, ws, nv = _decode(c, logical, masks=masks)
+    b_out, b_lse, b_w = brute.dense_attention(c["q"][-1:], c["pool"], c["bt"], c["L"], logical, 1,
+                                              visible_tokens=tokens)
+    np.testing.assert_allclose(out, b_out, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(lse, b_lse, rtol=1e-11)
+    np.testing.assert_allclose(ws, 1.0, rtol=1e-12)
+    assert np.all(nv == len(tokens))
+    hidden = np.ones(c["L"], dtype=bool)
+    hidden[sorted(tokens)] = False
+    assert np.all(b_w[0][:, hidden] == 0.0)
+    full = _decode(c, logical, masks=np.full(len(logical), 0xFFFF, dtype=np.uint16))
+    plain = _decode(c, logical)
+    for a, b in zip(full, plain):
+        assert np.array_equal(a, b)
+
+
+def test_token_mask_closed_form_and_planted_key():
+    """q = 0 under a token mask: lse = ln(#set bits inside the context) and out = mean of exactly
+    those value rows.  A dominant key at a token whose bit is clear leaves the result unchanged;
+    setting the bit makes the output that token's value row."""
+    c = _small_case(5, L=203)
+    logical = np.array([0, 2, 3, 7, c["n_pages"] - 1])
+    masks = np.array([0x0001, 0x8000, 0x0F0F, 0xFFFE, 0xFFFF], dtype=np.uint16)
+    tokens = [lp * P + t for lp, m in zip(logical, masks) for t in range(P)
+              if (int(m) >> t) & 1 and lp * P + t < c["L"]]
+    q0 = np.zeros_like(c["q"][-1:])
+    out, lse, _, nv = _decode(c, logical, q=q0, masks=masks)
+    assert np.all(nv == len(tokens))
+    np.testing.assert_allclose(lse, np.log(len(tokens)), rtol=1e-14)
+    pool = synth.bf16_bits_to_f64(c["pool"])
+    G = c["Hq"] // c["Hkv"]
+    for h in range(c["Hq"]):
+        rows = np.stack([pool[c["bt"][t // P], 1, h // G, t % P] for t in tokens])
+        np.testing.assert_allclose(out[0, h], rows.mean(0), rtol=1e-12, atol=1e-14)
+    # planted key at token 7*P + 0 (bit 0 of mask 0xFFFE is clear)
+    head, token = 3, 7 * P
+    planted = c["pool"].copy()
+    _plant_key(c, planted, token, c["q"][-1], head)
+    base = _decode(c, logical, masks=masks)
+    hidden = _decode(c, logical, pool=planted, masks=masks)
+    np.testing.assert_array_equal(hidden[0][0, head], base[0][0, head])
+    masks_on = masks.copy()
+    masks_on[3] = 0xFFFF
+    seen = _decode(c, logical, pool=planted, masks=masks_on)
+    v_row = synth.bf16_bits_to_f64(planted)[c["bt"][7], 1, head // G, 0]
+    np.testing.assert_allclose(seen[0][0, head], v_row, atol=1e-9)
 
 
 def test_uniform_attention_closed_form():
