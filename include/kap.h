@@ -78,11 +78,16 @@ enum {
  *      logical order; plan_phys_pages[i] = bt_pages[bt_indptr[b] + plan_logical_pages[i]].
  *   5. force_full[b] != 0 selects every page and sets KAP_PLAN_FULL (the fallback path, Section 3.2
  *      "Runtime stability and fallback"); selected/total pages > s_max sets KAP_PLAN_S_HIGH.
+ *   6. plan_token_masks (optional, page_size <= 16): one 16-bit word per listed page, bit t set
+ *      iff token page * page_size + t belongs to the selected union U.  It is the plan's visibility
+ *      mask (Section 3.1 "Selected-KV view materialization") at token granularity; without it the
+ *      attention call treats every token of a listed page as visible.
  *
  * plan_indptr[batch+1], plan_flags[batch] and selected_tokens[batch] (may be NULL) are written;
  * plan_logical_pages / plan_phys_pages receive plan_indptr[batch] entries and must hold
  * plan_capacity entries.  plan_phys_pages may be NULL; it requires a block table otherwise.
- * force_full and the block table may be NULL.
+ * force_full and the block table may be NULL.  plan_token_masks may be NULL; it must hold
+ * plan_capacity entries otherwise (KAP_ERR_UNSUPPORTED when page_size > 16).
  *
  * Errors: KAP_ERR_INVALID_ARG for batch < 0, page_size <= 0, ctx_len <= 0, a negative budget /
  * sink / recent / span length, a NaN score, a non-monotone span_indptr, a block table shorter than
@@ -109,7 +114,8 @@ kap_status kap_compile_plan(
     int32_t* plan_logical_pages,       /* HOST out, ascending per sequence */
     int32_t* plan_phys_pages,          /* HOST out or NULL */
     int32_t* plan_flags,               /* HOST out [batch] */
-    int32_t* selected_tokens);         /* HOST out [batch] or NULL: size of the token union */
+    int32_t* selected_tokens,          /* HOST out [batch] or NULL: size of the token union */
+    uint16_t* plan_token_masks);       /* HOST out or NULL: per listed page, bit t = token t selected */
 
 /*
  * Workspace: the split-K work list of one launch shape and the buffers for the partial results
@@ -174,6 +180,10 @@ kap_status kap_schedule_info(const kap_workspace* ws, int32_t* n_items, int32_t*
  * softmax); the splits' results are merged by log-sum-exp, inside a thread-block cluster through
  * distributed shared memory and, for lists too long for one cluster, by a separate merge pass.  One layer per call.
  * plan_logical_pages == NULL means "logical page = position in the list" (identity plan).
+ * plan_token_masks == NULL means every token of a listed page is visible (page-granular view:
+ * the page is read whole either way).  With masks, Vis(b) shrinks to the tokens whose bit is set
+ * (still t < ctx_len[b]); masked tokens get weight exactly 0, and a head that sees no token at all
+ * returns out = 0 and lse = -inf.  The bytes read do not change.
  * The plan arrays are the DEVICE copies of kap_compile_plan's outputs; `ws` must hold a schedule
  * made from the same per-sequence list lengths with n_q = NULL.
  * Errors: KAP_ERR_INVALID_ARG (NULL pointer, batch mismatch with the schedule, misaligned pool),
@@ -186,6 +196,7 @@ kap_status kap_selected_decode_attn(
     const int32_t* plan_indptr,        /* DEVICE [batch+1] */
     const int32_t* plan_phys_pages,    /* DEVICE [plan_indptr[batch]] */
     const int32_t* plan_logical_pages, /* DEVICE same length, or NULL */
+    const uint16_t* plan_token_masks,  /* DEVICE same length, or NULL */
     const int32_t* ctx_len,            /* DEVICE [batch] */
     int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
     float sm_scale,

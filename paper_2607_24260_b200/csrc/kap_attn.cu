@@ -45,13 +45,14 @@ constexpr int kDefaultSlots = 8;                          // 8 slots -> 3 CTAs/S
 constexpr int kHalfTileBytes = kPageSize * 128;           // 16 tokens x 64 bf16 = 2048 B
 constexpr int kTileBytes = 2 * kHalfTileBytes;            // K (or V) of one page and head: 4096 B
 constexpr int kPageHeadBytes = 2 * kTileBytes;            // K + V: 8192 B
-constexpr int kMaxIds = 768;                              // page ids a CTA can hold (dynamic sharing up to this)
+constexpr int kMaxIds = 640;                              // page ids a CTA can hold (dynamic sharing up to this)
 constexpr int kScratchStride = kHeadDim + 8;              // floats per scratch row (bank spread)
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;         // per-CTA deadline for all waits
 
 struct SmemTail {                                         // control block in front of the ring
     int32_t phys[kMaxIds];
     int32_t logical[kMaxIds];
+    uint16_t mask[kMaxIds];                   // token-visibility bits of each page (all ones: whole page)
     int32_t slot_page[kMaxSlots];             // list index of the page in each ring slot, -1 = no more
     uint32_t slot_done[kMaxSlots];            // warps that have finished with the slot's current page
     unsigned long long full[kMaxSlots];
@@ -62,6 +63,7 @@ struct SmemTail {                                         // control block in fr
     int32_t timed_out;
 };
 constexpr int kTailBytes = ((int)sizeof(SmemTail) + 1023) / 1024 * 1024;   // the ring follows, 1 KiB aligned
+static_assert(kTailBytes == 8192, "control block must stay within 8 KiB: 3 CTAs per SM with an 8-slot ring");
 constexpr int smem_bytes_for(int slots) { return kTailBytes + slots * kPageHeadBytes + 1024; }  // + alignment slack
 
 static_assert(kWarps * kRowTile * kScratchStride * 4 <= kDefaultSlots * kPageHeadBytes,
@@ -73,6 +75,7 @@ struct AttnParams {
     const int32_t* list_indptr;      // [B+1]
     const int32_t* phys_pages;
     const int32_t* logical_pages;    // or null: logical page = position in the list
+    const uint16_t* token_masks;     // or null: every token of a listed page is visible
     const int32_t* ctx_len;          // [B]
     const WorkItem* items;
     const MergeGroup* groups;
@@ -313,6 +316,7 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         if (!ok) { ph = 0; atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX); }
         tail->phys[i] = ph;
         tail->logical[i] = p.logical_pages && ok ? p.logical_pages[list0 + i] : item.page_begin + i;
+        tail->mask[i] = p.token_masks && ok ? p.token_masks[list0 + i] : (uint16_t)0xFFFFu;
     }
     __syncthreads();
     KAP_TRACE_POINT(blockIdx.x, 1);
@@ -437,14 +441,16 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             mma_bf16(sacc[0], qf[ks], b0, b1);
             mma_bf16(sacc[1], qf[ks], b2, b3);
         }
-        if (tok0 + kPageSize - 1 > full_vis_limit) {
-            // page reaches into the causal / tail region: mask per element
+        const uint32_t tmask = tail->mask[page];
+        if (tok0 + kPageSize - 1 > full_vis_limit || tmask != 0xFFFFu) {
+            // page reaches into the causal / tail region, or only some of its tokens are in the
+            // selected union: mask per element
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int t = tok0 + nt * 8 + tid4 * 2 + (e & 1);
-                    if (t > pos_row[e >> 1]) sacc[nt][e] = -INFINITY;
+                    const int slot = nt * 8 + tid4 * 2 + (e & 1);
+                    if (tok0 + slot > pos_row[e >> 1] || !((tmask >> slot) & 1u)) sacc[nt][e] = -INFINITY;
                 }
             // value rows past the end of the context may hold anything (even NaN): zero them
             const int first_bad = L - tok0;
@@ -968,7 +974,8 @@ static AttnParams base_params(kap_workspace* ws, int32_t hq, int32_t hkv, float 
 
 extern "C" kap_status kap_selected_decode_attn(
     const void* q, const void* kv_pool, int64_t num_pool_pages, const int32_t* plan_indptr,
-    const int32_t* plan_phys_pages, const int32_t* plan_logical_pages, const int32_t* ctx_len,
+    const int32_t* plan_phys_pages, const int32_t* plan_logical_pages,
+    const uint16_t* plan_token_masks, const int32_t* ctx_len,
     int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
     float sm_scale, void* out, float* lse, kap_workspace* ws, void* cuda_stream)
 {
@@ -980,6 +987,7 @@ extern "C" kap_status kap_selected_decode_attn(
     AttnParams p = base_params(ws, num_q_heads, num_kv_heads, sm_scale, num_pool_pages);
     p.q = (const __nv_bfloat16*)q; p.q_indptr = nullptr; p.list_indptr = plan_indptr;
     p.phys_pages = plan_phys_pages; p.logical_pages = plan_logical_pages; p.ctx_len = ctx_len;
+    p.token_masks = plan_token_masks;
     p.out = (__nv_bfloat16*)out; p.lse = lse;
     return launch_attention(p, kv_pool, num_pool_pages, ws, (cudaStream_t)cuda_stream);
 }

@@ -73,7 +73,8 @@ extern "C" kap_status kap_compile_plan(
     const int32_t* budget_tokens, const int32_t* n_sink, const int32_t* n_recent,
     const uint8_t* force_full, float s_max, const int32_t* bt_indptr, const int32_t* bt_pages,
     int64_t plan_capacity, int32_t* plan_indptr, int32_t* plan_logical_pages,
-    int32_t* plan_phys_pages, int32_t* plan_flags, int32_t* selected_tokens)
+    int32_t* plan_phys_pages, int32_t* plan_flags, int32_t* selected_tokens,
+    uint16_t* plan_token_masks)
 {
     using namespace kap;
     if (batch < 0) return fail(KAP_ERR_INVALID_ARG, "batch %d < 0", batch);
@@ -86,6 +87,8 @@ extern "C" kap_status kap_compile_plan(
         return fail(KAP_ERR_INVALID_ARG, "block table needs both bt_indptr and bt_pages");
     if (plan_phys_pages && !bt_indptr)
         return fail(KAP_ERR_INVALID_ARG, "plan_phys_pages requested without a block table");
+    if (plan_token_masks && page_size > 16)
+        return fail(KAP_ERR_UNSUPPORTED, "token masks hold 16 bits per page, page_size is %d", page_size);
     if (std::isnan(s_max)) return fail(KAP_ERR_INVALID_ARG, "s_max is NaN");
     if (batch > 0 && span_indptr[0] != 0)
         return fail(KAP_ERR_INVALID_ARG, "span_indptr[0] = %d, expected 0", span_indptr[0]);
@@ -117,6 +120,7 @@ extern "C" kap_status kap_compile_plan(
     // ---- selection pass, into temporaries
     std::vector<int32_t> indptr(batch + 1, 0), flags(batch, 0), used_tokens(batch, 0);
     std::vector<int32_t> logical;
+    std::vector<uint16_t> masks;
     std::vector<Interval> u;
     std::vector<Candidate> cand;
     for (int32_t b = 0; b < batch; ++b) {
@@ -165,6 +169,21 @@ extern "C" kap_status kap_compile_plan(
             for (int32_t p = p0; p <= p1; ++p) { logical.push_back(p); ++n_sel; }
             last_page = std::max(last_page, p1);
         }
+        if (plan_token_masks) {
+            // bit t of a listed page: token page*P + t lies in the union (intervals and pages both
+            // ascend, so one forward sweep pairs them up)
+            masks.resize(logical.size(), 0);
+            size_t e = (size_t)indptr[b];
+            for (const auto& iv : u) {
+                while ((int64_t)logical[e] * page_size + page_size <= iv.lo) ++e;
+                for (size_t k = e; k < logical.size() && (int64_t)logical[k] * page_size < iv.hi; ++k) {
+                    const int64_t base = (int64_t)logical[k] * page_size;
+                    const int lo = (int)std::max<int64_t>(iv.lo - base, 0);
+                    const int hi = (int)std::min<int64_t>(iv.hi - base, page_size);
+                    masks[k] |= (uint16_t)(((1u << hi) - 1u) & ~((1u << lo) - 1u));
+                }
+            }
+        }
         if ((double)n_sel / (double)n_pages > (double)s_max) fl |= KAP_PLAN_S_HIGH;
         if ((int64_t)logical.size() > (int64_t)INT32_MAX)
             return fail(KAP_ERR_CAPACITY, "plan exceeds 2^31 pages");
@@ -184,6 +203,8 @@ extern "C" kap_status kap_compile_plan(
         for (int32_t b = 0; b < batch; ++b)
             for (int32_t i = indptr[b]; i < indptr[b + 1]; ++i)
                 plan_phys_pages[i] = bt_pages[bt_indptr[b] + logical[i]];
+    if (plan_token_masks && !masks.empty())
+        std::memcpy(plan_token_masks, masks.data(), sizeof(uint16_t) * masks.size());
     for (int32_t b = 0; b < batch; ++b) {
         plan_flags[b] = flags[b];
         if (selected_tokens) selected_tokens[b] = used_tokens[b];

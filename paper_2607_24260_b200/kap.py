@@ -23,7 +23,7 @@ _i32p, _f32p, _u8p, _vp = C.POINTER(C.c_int32), C.POINTER(C.c_float), C.POINTER(
 SIGNATURES = {
     "kap_compile_plan": (C.c_int, [C.c_int32, C.c_int32, _i32p, _i32p, _i32p, _i32p, _f32p, _i32p,
                                    _i32p, _i32p, _u8p, C.c_float, _i32p, _i32p, C.c_int64, _i32p,
-                                   _i32p, _i32p, _i32p, _i32p]),
+                                   _i32p, _i32p, _i32p, _i32p, C.POINTER(C.c_uint16)]),
     "kap_workspace_create": (C.c_int, [C.POINTER(_vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
     "kap_workspace_destroy": (None, [_vp]),
     "kap_schedule": (C.c_int, [_vp, C.c_int32, _i32p, _i32p, C.c_int32, C.c_int32, C.c_int32, _vp]),
@@ -31,7 +31,7 @@ SIGNATURES = {
                                     C.c_int32, C.c_int32, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                     _i32p]),
     "kap_schedule_info": (C.c_int, [_vp, _i32p, _i32p, _i32p, _i32p, _i32p]),
-    "kap_selected_decode_attn": (C.c_int, [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, C.c_int32,
+    "kap_selected_decode_attn": (C.c_int, [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp, _vp, C.c_int32,
                                            C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float,
                                            _vp, _vp, _vp, _vp]),
     "kap_verify_attn": (C.c_int, [_vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_int32, C.c_int32,
@@ -109,7 +109,9 @@ def compile_plan(ctx_len, span_indptr, span_start, span_len, span_score, budget_
                  n_recent, force_full=None, s_max=1.0, bt_indptr=None, bt_pages=None, page_size=16,
                  capacity=None):
     """kap_compile_plan on host arrays.  Returns a dict: plan_indptr, plan_logical_pages,
-    plan_phys_pages (None without a block table), plan_flags, selected_tokens."""
+    plan_phys_pages (None without a block table), plan_flags, selected_tokens, plan_token_masks
+    (uint16 per listed page, bit t = token t of the page is in the selected union; None when
+    page_size > 16)."""
     ctx_len = _np(ctx_len, np.int32)
     B = int(ctx_len.shape[0])
     span_indptr, span_start = _np(span_indptr, np.int32), _np(span_start, np.int32)
@@ -124,17 +126,20 @@ def compile_plan(ctx_len, span_indptr, span_start, span_len, span_score, budget_
     phys = np.full(max(1, capacity), -1, dtype=np.int32) if bt_indptr is not None else None
     flags = np.full(B, -1, dtype=np.int32)
     sel = np.full(B, -1, dtype=np.int32)
+    masks = np.zeros(max(1, capacity), dtype=np.uint16) if 0 < page_size <= 16 else None
     _check(lib().kap_compile_plan(
         B, page_size, _ptr(ctx_len, C.c_int32), _ptr(span_indptr, C.c_int32),
         _ptr(span_start, C.c_int32), _ptr(span_len, C.c_int32), _ptr(span_score, C.c_float),
         _ptr(budget_tokens, C.c_int32), _ptr(n_sink, C.c_int32), _ptr(n_recent, C.c_int32),
         _ptr(force_full, C.c_uint8), float(s_max), _ptr(bt_indptr, C.c_int32),
         _ptr(bt_pages, C.c_int32), int(capacity), _ptr(indptr, C.c_int32), _ptr(logical, C.c_int32),
-        _ptr(phys, C.c_int32), _ptr(flags, C.c_int32), _ptr(sel, C.c_int32)))
+        _ptr(phys, C.c_int32), _ptr(flags, C.c_int32), _ptr(sel, C.c_int32),
+        _ptr(masks, C.c_uint16)))
     n = int(indptr[-1])
     return dict(plan_indptr=indptr, plan_logical_pages=logical[:n].copy(),
                 plan_phys_pages=None if phys is None else phys[:n].copy(), plan_flags=flags,
-                selected_tokens=sel)
+                selected_tokens=sel,
+                plan_token_masks=None if masks is None else masks[:n].copy())
 
 
 def compile_workload(w, capacity=None):
@@ -209,16 +214,17 @@ class Workspace:
 
 
 def selected_decode_attn(q, kv_pool, plan_indptr, plan_phys_pages, plan_logical_pages, ctx_len, out,
-                         ws: Workspace, lse=None, sm_scale=None, stream=None):
+                         ws: Workspace, lse=None, sm_scale=None, stream=None, plan_token_masks=None):
     """kap_selected_decode_attn on torch CUDA tensors: q/out bf16 [B, Hq, d]; kv_pool bf16
-    [pages, 2, Hkv, P, d]; plan arrays and ctx_len int32 device tensors."""
+    [pages, 2, Hkv, P, d]; plan arrays and ctx_len int32 device tensors; plan_token_masks an
+    optional uint16 device tensor (one word per listed page) for token-granular visibility."""
     B, Hq, d = q.shape
     pages, _, Hkv, P, _ = kv_pool.shape
     sm_scale = float(d) ** -0.5 if sm_scale is None else float(sm_scale)
     _check(lib().kap_selected_decode_attn(
         _dptr(q), _dptr(kv_pool), int(pages), _dptr(plan_indptr), _dptr(plan_phys_pages),
-        _dptr(plan_logical_pages), _dptr(ctx_len), B, Hq, Hkv, d, P, sm_scale, _dptr(out),
-        _dptr(lse), ws._h, _stream_ptr(stream)))
+        _dptr(plan_logical_pages), _dptr(plan_token_masks), _dptr(ctx_len), B, Hq, Hkv, d, P,
+        sm_scale, _dptr(out), _dptr(lse), ws._h, _stream_ptr(stream)))
     return out
 
 

@@ -28,10 +28,16 @@ def i32(a) -> torch.Tensor:
     return torch.from_numpy(np.array(a, dtype=np.int32, copy=True)).to(DEV)
 
 
+def u16(a) -> torch.Tensor:
+    """uint16 words -> device tensor of the same bits (carried as int16)."""
+    return torch.from_numpy(np.array(a, dtype=np.uint16, copy=True).view(np.int16)).to(DEV)
+
+
 def run_decode(q_bits, pool_dev, plan, ctx_len, Hq=32, Hkv=8, max_chunk_pages=0, ws=None,
-               logical=True, sm_scale=None):
+               logical=True, sm_scale=None, masks=None):
     """Library proposal-path attention.  q_bits [B, Hq, d] uint16; pool_dev torch bf16
-    [pages, 2, Hkv, P, d]; plan = dict from a plan compiler.  Returns (out f64, lse f64)."""
+    [pages, 2, Hkv, P, d]; plan = dict from a plan compiler; masks = optional uint16 word per
+    listed page (token-granular visibility).  Returns (out f64, lse f64)."""
     B = q_bits.shape[0]
     n = np.diff(plan["plan_indptr"])
     own = ws is None
@@ -43,7 +49,8 @@ def run_decode(q_bits, pool_dev, plan, ctx_len, Hq=32, Hkv=8, max_chunk_pages=0,
     lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV)
     kap.selected_decode_attn(q, pool_dev, i32(plan["plan_indptr"]), i32(plan["plan_phys_pages"]),
                              i32(plan["plan_logical_pages"]) if logical else None, i32(ctx_len),
-                             out, ws, lse=lse, sm_scale=sm_scale)
+                             out, ws, lse=lse, sm_scale=sm_scale,
+                             plan_token_masks=None if masks is None else u16(masks))
     ws.check()
     res = dev_bf16_to_f64(out), lse.double().cpu().numpy()
     if own:
@@ -75,10 +82,10 @@ def run_verify(q_bits, n_q, pool_dev, bt_indptr, bt_pages, ctx_len, Hq=32, Hkv=8
     return res
 
 
-def oracle_decode(q_bits, pool_bits, plan, ctx_len, scale=None):
+def oracle_decode(q_bits, pool_bits, plan, ctx_len, scale=None, masks=None):
     out, lse, _, _ = orc.selected_decode_attn(q_bits, pool_bits, plan["plan_indptr"],
                                               plan["plan_phys_pages"], plan["plan_logical_pages"],
-                                              ctx_len, scale=scale)
+                                              ctx_len, scale=scale, plan_token_masks=masks)
     return out, lse
 
 

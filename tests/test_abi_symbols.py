@@ -57,8 +57,9 @@ int main(void) {
     int32_t budget[1] = {48}, sink[1] = {4}, recent[1] = {8};
     int32_t bt_indptr[2] = {0, 7}, bt[7] = {17, 3, 9, 12, 5, 30, 2};
     int32_t out_indptr[2], logical[7], phys[7], flags[1], sel[1];
+    uint16_t masks[7];
     kap_status st = kap_compile_plan(1, 16, ctx, indptr, start, len, score, budget, sink, recent, 0, 1.0f,
-                                     bt_indptr, bt, 7, out_indptr, logical, phys, flags, sel);
+                                     bt_indptr, bt, 7, out_indptr, logical, phys, flags, sel, masks);
     if (st != KAP_OK) { printf("error %d: %s\n", (int)st, kap_last_error()); return 1; }
     printf("%s |", kap_version());
     for (int i = 0; i < out_indptr[1]; ++i) printf(" %d:%d", logical[i], phys[i]);

@@ -7,7 +7,16 @@ from helpers import read_plan_fixture
 from oracle import kap_oracle as orc
 from paper_2607_24260_b200 import kap, synth
 
-KEYS = ("plan_indptr", "plan_logical_pages", "plan_phys_pages", "plan_flags", "selected_tokens")
+KEYS = ("plan_indptr", "plan_logical_pages", "plan_phys_pages", "plan_flags", "selected_tokens",
+        "plan_token_masks")
+
+
+def _same(a, b, msg=""):
+    if a is None or b is None:
+        assert a is None and b is None, msg
+    else:
+        assert a.dtype == b.dtype, msg
+        np.testing.assert_array_equal(a, b, err_msg=msg)
 
 
 def test_fixture_through_the_library():
@@ -29,7 +38,8 @@ def test_library_equals_oracle_on_random_tiny_cases():
                               page_size=(16, 4, 1, 32)[seed % 4])
         a, b = kap.compile_workload(w), orc.compile_workload(w)
         for k in KEYS:
-            np.testing.assert_array_equal(a[k], b[k], err_msg=f"seed {seed} {k}")
+            _same(a[k], b[k], f"seed {seed} {k}")
+        assert (a["plan_token_masks"] is None) == (w.page_size > 16)
 
 
 @pytest.mark.parametrize("name", ["c1", "c1b", "c2", "c3", "c4", "c5"])
@@ -37,7 +47,11 @@ def test_library_equals_oracle_on_the_named_configs(name):
     w = synth.CONFIGS[name](0)
     a, b = kap.compile_workload(w), orc.compile_workload(w)
     for k in KEYS:
-        np.testing.assert_array_equal(a[k], b[k])
+        _same(a[k], b[k], k)
+    # the masks count exactly the selected tokens
+    bits = np.array([bin(int(m)).count("1") for m in a["plan_token_masks"]])
+    per_seq = np.add.reduceat(bits, a["plan_indptr"][:-1])
+    np.testing.assert_array_equal(per_seq, a["selected_tokens"])
     # retained ratio s (Eq. 4, in pages) lands near the stated budgets
     s = np.diff(a["plan_indptr"]) / ((w.ctx_len + 15) // 16)
     if name == "c4":
@@ -91,13 +105,13 @@ def test_capacity_error_and_untouched_outputs():
     bud = np.array([64, 64], dtype=np.int32)
     rc = kap.lib().kap_compile_plan(2, 16, p(ctx), p(np.zeros(3, dtype=np.int32)), None, None, None,
                                     p(bud), p(sink), p(z), None, 1.0, None, None, 4, p(indptr),
-                                    p(pages), None, p(flags), None)
+                                    p(pages), None, p(flags), None, None)
     assert rc == kap.ERR_CAPACITY                  # 8 pages needed, 4 offered
     assert np.all(indptr == -7) and np.all(pages == -7) and np.all(flags == -7)
     pages = np.full(8, -7, dtype=np.int32)
     rc = kap.lib().kap_compile_plan(2, 16, p(ctx), p(np.zeros(3, dtype=np.int32)), None, None, None,
                                     p(bud), p(sink), p(z), None, 1.0, None, None, 8, p(indptr),
-                                    p(pages), None, p(flags), None)
+                                    p(pages), None, p(flags), None, None)
     assert rc == kap.OK and indptr.tolist() == [0, 4, 8] and pages.tolist() == [0, 1, 2, 3] * 2
 
 
