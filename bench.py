@@ -383,6 +383,36 @@ def time_extras(cy: Cycle, vocab: int = 128256, iters: int = 20):
     us = timed(view)
     out["materialize_view_us_per_layer"] = us
     out["materialize_view_GBps_read_plus_write"] = 2 * n * w.page_bytes / (us * 1e-6) / 1e9
+    # growing plan: compiled once, recent-window entries refreshed on the device every step, the
+    # proposal kernel run with token-granular masks (a different layer each call)
+    t0 = time.perf_counter()
+    for _ in range(iters):
+        grow = kap.compile_growing_plan(w.ctx_len, w.span_indptr, w.span_start, w.span_len, w.span_score,
+                                        w.budget_tokens, w.n_sink, w.n_recent, w.bt_indptr, w.bt_pages,
+                                        force_full=w.force_full, max_growth=4096)
+    out["compile_growing_plan_ms"] = (time.perf_counter() - t0) / iters * 1e3
+    i32 = lambda a: torch.from_numpy(np.array(a, dtype=np.int32, copy=True)).to(dev)
+    g_indptr, g_phys, g_logical = i32(grow["plan_indptr"]), i32(grow["plan_phys_pages"]), i32(grow["plan_logical_pages"])
+    g_masks = torch.from_numpy(np.array(grow["plan_token_masks"], copy=True).view(np.int16)).to(dev)
+    g_tail = i32(grow["tail_desc"])
+    ws = kap.Workspace(int(dev.split(":")[1]), 8192, w.num_q_heads // w.num_kv_heads, w.batch)
+    ws.schedule(np.diff(grow["plan_indptr"]), None, w.num_q_heads, w.num_kv_heads)
+    out["refresh_recent_us"] = timed(lambda: kap.refresh_recent(
+        g_indptr, g_logical, g_phys, g_masks, g_tail, cy.d_bt_indptr, cy.d_bt_pages, cy.d_ctx,
+        w.num_pool_pages))
+    o = torch.empty_like(cy.q_dec[0, 0])
+
+    def masked():
+        layer = turn[0] % cy.layers
+        kap.selected_decode_attn(cy.q_dec[0, layer], cy.pool[layer], g_indptr, g_phys, g_logical, cy.d_ctx,
+                                 o, ws, plan_token_masks=g_masks)
+        turn[0] += 1
+    kap.refresh_recent(g_indptr, g_logical, g_phys, g_masks, g_tail, cy.d_bt_indptr, cy.d_bt_pages, cy.d_ctx,
+                       w.num_pool_pages)
+    torch.cuda.synchronize()
+    out["growing_plan_decode_us_per_layer"] = timed(masked)
+    ws.check()
+    ws.close()
     return out
 
 

@@ -58,7 +58,9 @@ typedef enum {
 enum {
     KAP_PLAN_FULL = 1,         /* identity plan: the sequence takes full-context access */
     KAP_PLAN_OVER_BUDGET = 2,  /* the mandatory tokens alone exceed the budget; no span selected */
-    KAP_PLAN_S_HIGH = 4        /* retained ratio s (Eq. 4, in pages) > s_max: caller should fall back */
+    KAP_PLAN_S_HIGH = 4,       /* retained ratio s (Eq. 4, in pages) > s_max: caller should fall back */
+    KAP_PLAN_MOVES_WITH_LENGTH = 8  /* growing plans only: compiled at another length, Algorithm 1
+                                       could have selected other spans (see kap_compile_growing_plan) */
 };
 
 /*
@@ -311,6 +313,76 @@ kap_status kap_top3_accept(
  */
 kap_status kap_phase_model(double k, double h, double s, double w_main, double w_prop, double kv,
                            double* out /* HOST [8] */);
+
+/*
+ * kap_compile_growing_plan / kap_refresh_recent - one compiled plan for a context that grows
+ * (Section 3.2: k proposal steps per cycle, many cycles per request; the plan is compiled once per
+ * request, Section 3.1).  The selected union U of Algorithm 1 has a part that does not depend on
+ * the length - the sink prefix and the selected spans - and the recent window [L - n_recent, L)
+ * (at least the last token), which moves.  kap_compile_growing_plan runs Algorithm 1 exactly as
+ * kap_compile_plan does (same arguments, same ranking, same budget accounting at ctx_len) but
+ * lists, per sequence, the pages and token masks of the fixed part followed by reserved entries
+ * with empty masks; kap_refresh_recent, a small kernel, rewrites the reserved entries from the
+ * device-side ctx_len: the window's pages, with masks that omit tokens the fixed part already
+ * lists.  kap_selected_decode_attn on these arrays (plan_token_masks is required) then sees
+ * exactly fixed part + window at the current length, and one kap_schedule (list lengths never
+ * change) serves every step.  A page that holds both fixed and window tokens is listed twice with
+ * disjoint masks; an entry with an empty mask is neither fetched nor computed.
+ *
+ * A full-context plan (force_full) lists the whole prefix and reserves entries for every token
+ * from ctx_len on, up to max_growth more tokens; for other sequences max_growth is not needed.
+ *
+ * When is this the plan Algorithm 1 would compile at the longer length?  Whenever the sink and
+ * every non-empty span end at or before ctx_len - max(n_recent, 1): then no span shares tokens
+ * with the window at this or any greater length and span costs do not change.  Otherwise the
+ * sequence gets KAP_PLAN_MOVES_WITH_LENGTH: the arrays are still valid (fixed part + window, no
+ * token twice) but a fresh compile could select other spans.
+ *
+ * tail_desc[b] = { reserved entries, window tokens (INT32_MAX: everything), first token the
+ * reserved entries may cover }; copy it to the device for kap_refresh_recent.  selected_tokens and
+ * the flags describe the plan at ctx_len.  The reserved entries start out empty: call
+ * kap_refresh_recent before the first attention call.
+ * Errors of kap_compile_growing_plan: as kap_compile_plan, plus KAP_ERR_INVALID_ARG for
+ * max_growth < 0, a missing block table, or a NULL plan_phys_pages / plan_token_masks / tail_desc.
+ *
+ * kap_refresh_recent: DEVICE pointers; asynchronous on cuda_stream; captured into CUDA graphs
+ * like the attention calls.  Problems found on the device (a window page without a block-table
+ * entry, a page outside the pool, a context that outgrew the reservation, ctx_len <= 0) set
+ * 1 << KAP_ERR_DEVICE_INDEX in *device_status, or in the status word of `ws` when device_status is
+ * NULL, and leave the affected entries empty.  `ws` (may be NULL) is the workspace of the
+ * attention call that will read the arrays: its next launch is then issued without programmatic
+ * dependent launch, because the attention prologue reads the lists ahead of the dependency wait.
+ * Errors: KAP_ERR_UNSUPPORTED (page_size > 16), KAP_ERR_INVALID_ARG, KAP_ERR_CUDA.
+ */
+kap_status kap_compile_growing_plan(
+    int32_t batch, int32_t page_size,
+    const int32_t* ctx_len, const int32_t* span_indptr, const int32_t* span_start,
+    const int32_t* span_len, const float* span_score, const int32_t* budget_tokens,
+    const int32_t* n_sink, const int32_t* n_recent, const uint8_t* force_full, float s_max,
+    const int32_t* bt_indptr, const int32_t* bt_pages,   /* HOST, as kap_compile_plan; required */
+    int32_t max_growth,                /* tokens a full-context sequence may still grow by */
+    int64_t plan_capacity,
+    int32_t* plan_indptr,              /* HOST out [batch+1], reserved entries included */
+    int32_t* plan_logical_pages,       /* HOST out */
+    int32_t* plan_phys_pages,          /* HOST out */
+    uint16_t* plan_token_masks,        /* HOST out */
+    int32_t* plan_flags,               /* HOST out [batch] */
+    int32_t* selected_tokens,          /* HOST out [batch] or NULL */
+    int32_t* tail_desc);               /* HOST out [batch][3] */
+
+kap_status kap_refresh_recent(
+    const int32_t* plan_indptr,        /* DEVICE [batch+1] */
+    int32_t* plan_logical_pages,       /* DEVICE in/out */
+    int32_t* plan_phys_pages,          /* DEVICE in/out */
+    uint16_t* plan_token_masks,        /* DEVICE in/out */
+    const int32_t* tail_desc,          /* DEVICE [batch][3] */
+    const int32_t* bt_indptr,          /* DEVICE [batch+1] */
+    const int32_t* bt_pages,           /* DEVICE */
+    const int32_t* ctx_len,            /* DEVICE [batch] current lengths */
+    int32_t batch, int32_t page_size, int64_t num_pool_pages,
+    int32_t* device_status,            /* DEVICE or NULL */
+    kap_workspace* ws,                 /* or NULL */
+    void* cuda_stream);
 
 /*
  * kap_materialize_view - the paper's selected-KV view as a physical copy (Section 3.1,

@@ -338,6 +338,10 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         const int idx = first_idx + k * idx_stride;
         if (idx < n_pages) {
             tail->slot_page[s] = idx;
+            if (tail->mask[idx] == 0) {                      // no visible token: nothing to fetch
+                mbar_arrive(bar);
+                return;
+            }
             const int y = tail->phys[idx] * rows_per_page + item.kv_head * kPageSize;
             const uint32_t dst = smem_u32(ring + s * kPageHeadBytes);
             mbar_expect_tx(bar, kPageHeadBytes);
@@ -427,83 +431,85 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         if (i == 0) KAP_TRACE_POINT(blockIdx.x, 3);
         const int page = tail->slot_page[s];
         if (page < 0 || tail->timed_out) break;              // the list is exhausted
-        const uint32_t kb = smem_u32(ring + s * kPageHeadBytes);
-        const uint32_t vb = kb + kTileBytes;
-        const int tok0 = tail->logical[page] * kPageSize;
-
-        // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
-        float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            uint32_t b0, b1, b2, b3;
-            ldsm_x4(kb + (ks >> 2) * kHalfTileBytes + k_tok * 128
-                       + ((((ks & 3) * 2 + k_cbit) ^ lr) << 4), b0, b1, b2, b3);
-            mma_bf16(sacc[0], qf[ks], b0, b1);
-            mma_bf16(sacc[1], qf[ks], b2, b3);
-        }
         const uint32_t tmask = tail->mask[page];
-        if (tok0 + kPageSize - 1 > full_vis_limit || tmask != 0xFFFFu) {
-            // page reaches into the causal / tail region, or only some of its tokens are in the
-            // selected union: mask per element
+        if (tmask != 0u) {                                   // a page without a visible token was not fetched
+            const uint32_t kb = smem_u32(ring + s * kPageHeadBytes);
+            const uint32_t vb = kb + kTileBytes;
+            const int tok0 = tail->logical[page] * kPageSize;
+
+            // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
+            float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int slot = nt * 8 + tid4 * 2 + (e & 1);
-                    if (tok0 + slot > pos_row[e >> 1] || !((tmask >> slot) & 1u)) sacc[nt][e] = -INFINITY;
-                }
-            // value rows past the end of the context may hold anything (even NaN): zero them
-            const int first_bad = L - tok0;
-            if (first_bad < kPageSize) {
-                if (lane < 16) {
-                    for (int r = max(first_bad, 0); r < kPageSize; ++r)
-                        *reinterpret_cast<uint4*>(ring + s * kPageHeadBytes + kTileBytes
-                                                  + (lane >> 3) * kHalfTileBytes + r * 128
-                                                  + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
+            for (int ks = 0; ks < 8; ++ks) {
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(kb + (ks >> 2) * kHalfTileBytes + k_tok * 128
+                           + ((((ks & 3) * 2 + k_cbit) ^ lr) << 4), b0, b1, b2, b3);
+                mma_bf16(sacc[0], qf[ks], b0, b1);
+                mma_bf16(sacc[1], qf[ks], b2, b3);
             }
-        }
-        // online softmax (base 2): rows gid (e = 0,1) and gid + 8 (e = 2,3)
-        float mx[2];
-        mx[0] = fmaxf(fmaxf(sacc[0][0], sacc[0][1]), fmaxf(sacc[1][0], sacc[1][1]));
-        mx[1] = fmaxf(fmaxf(sacc[0][2], sacc[0][3]), fmaxf(sacc[1][2], sacc[1][3]));
-        float corr[2], mu[2];
+            if (tok0 + kPageSize - 1 > full_vis_limit || tmask != 0xFFFFu) {
+                // page reaches into the causal / tail region, or only some of its tokens are in the
+                // selected union: mask per element
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
-            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-            const float mn = fmaxf(m_run[h], mx[h] * sc);
-            mu[h] = (mn == -INFINITY) ? 0.f : mn;
-            corr[h] = ex2(m_run[h] - mu[h]);
-            m_run[h] = mn;
-        }
-        uint32_t pa[4];      // P as the A operand of P V (rows gid / gid+8, tokens 0-7 / 8-15)
-        pa[0] = pack_bf16(ex2(fmaf(sacc[0][0], sc, -mu[0])), ex2(fmaf(sacc[0][1], sc, -mu[0])));
-        pa[1] = pack_bf16(ex2(fmaf(sacc[0][2], sc, -mu[1])), ex2(fmaf(sacc[0][3], sc, -mu[1])));
-        pa[2] = pack_bf16(ex2(fmaf(sacc[1][0], sc, -mu[0])), ex2(fmaf(sacc[1][1], sc, -mu[0])));
-        pa[3] = pack_bf16(ex2(fmaf(sacc[1][2], sc, -mu[1])), ex2(fmaf(sacc[1][3], sc, -mu[1])));
-        // the row sums use the rounded weights, so out = sum(p v) / sum(p) is a true average
-        l_run[0] = fmaf(l_run[0], corr[0],
-                        (bf16_lo(pa[0]) + bf16_hi(pa[0])) + (bf16_lo(pa[2]) + bf16_hi(pa[2])));
-        l_run[1] = fmaf(l_run[1], corr[1],
-                        (bf16_lo(pa[1]) + bf16_hi(pa[1])) + (bf16_lo(pa[3]) + bf16_hi(pa[3])));
-        if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+                for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-            for (int n = 0; n < 16; ++n) {
-                o[n][0] *= corr[0]; o[n][1] *= corr[0];
-                o[n][2] *= corr[1]; o[n][3] *= corr[1];
+                    for (int e = 0; e < 4; ++e) {
+                        const int slot = nt * 8 + tid4 * 2 + (e & 1);
+                        if (tok0 + slot > pos_row[e >> 1] || !((tmask >> slot) & 1u)) sacc[nt][e] = -INFINITY;
+                    }
+                // value rows past the end of the context may hold anything (even NaN): zero them
+                const int first_bad = L - tok0;
+                if (first_bad < kPageSize) {
+                    if (lane < 16) {
+                        for (int r = max(first_bad, 0); r < kPageSize; ++r)
+                            *reinterpret_cast<uint4*>(ring + s * kPageHeadBytes + kTileBytes
+                                                      + (lane >> 3) * kHalfTileBytes + r * 128
+                                                      + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                }
             }
-        }
-        // O += P V   (16 n-tiles of 8 output columns, two per ldmatrix)
+            // online softmax (base 2): rows gid (e = 0,1) and gid + 8 (e = 2,3)
+            float mx[2];
+            mx[0] = fmaxf(fmaxf(sacc[0][0], sacc[0][1]), fmaxf(sacc[1][0], sacc[1][1]));
+            mx[1] = fmaxf(fmaxf(sacc[0][2], sacc[0][3]), fmaxf(sacc[1][2], sacc[1][3]));
+            float corr[2], mu[2];
 #pragma unroll
-        for (int n2 = 0; n2 < 8; ++n2) {
-            uint32_t v0, v1, v2, v3;
-            ldsm_x4_t(vb + (n2 >> 2) * kHalfTileBytes + v_tok * 128
-                         + ((((n2 & 3) * 2 + v_cbit) ^ lr) << 4), v0, v1, v2, v3);
-            mma_bf16(o[2 * n2], pa, v0, v1);
-            mma_bf16(o[2 * n2 + 1], pa, v2, v3);
+            for (int h = 0; h < 2; ++h) {
+                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+                const float mn = fmaxf(m_run[h], mx[h] * sc);
+                mu[h] = (mn == -INFINITY) ? 0.f : mn;
+                corr[h] = ex2(m_run[h] - mu[h]);
+                m_run[h] = mn;
+            }
+            uint32_t pa[4];      // P as the A operand of P V (rows gid / gid+8, tokens 0-7 / 8-15)
+            pa[0] = pack_bf16(ex2(fmaf(sacc[0][0], sc, -mu[0])), ex2(fmaf(sacc[0][1], sc, -mu[0])));
+            pa[1] = pack_bf16(ex2(fmaf(sacc[0][2], sc, -mu[1])), ex2(fmaf(sacc[0][3], sc, -mu[1])));
+            pa[2] = pack_bf16(ex2(fmaf(sacc[1][0], sc, -mu[0])), ex2(fmaf(sacc[1][1], sc, -mu[0])));
+            pa[3] = pack_bf16(ex2(fmaf(sacc[1][2], sc, -mu[1])), ex2(fmaf(sacc[1][3], sc, -mu[1])));
+            // the row sums use the rounded weights, so out = sum(p v) / sum(p) is a true average
+            l_run[0] = fmaf(l_run[0], corr[0],
+                            (bf16_lo(pa[0]) + bf16_hi(pa[0])) + (bf16_lo(pa[2]) + bf16_hi(pa[2])));
+            l_run[1] = fmaf(l_run[1], corr[1],
+                            (bf16_lo(pa[1]) + bf16_hi(pa[1])) + (bf16_lo(pa[3]) + bf16_hi(pa[3])));
+            if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+                for (int n = 0; n < 16; ++n) {
+                    o[n][0] *= corr[0]; o[n][1] *= corr[0];
+                    o[n][2] *= corr[1]; o[n][3] *= corr[1];
+                }
+            }
+            // O += P V   (16 n-tiles of 8 output columns, two per ldmatrix)
+#pragma unroll
+            for (int n2 = 0; n2 < 8; ++n2) {
+                uint32_t v0, v1, v2, v3;
+                ldsm_x4_t(vb + (n2 >> 2) * kHalfTileBytes + v_tok * 128
+                             + ((((n2 & 3) * 2 + v_cbit) ^ lr) << 4), v0, v1, v2, v3);
+                mma_bf16(o[2 * n2], pa, v0, v1);
+                mma_bf16(o[2 * n2 + 1], pa, v2, v3);
+            }
         }
         // Done with the slot.  The last of the group's RT warps to get here refills it with the
         // group's page i + depth; nobody waits for anybody.  The fences order this warp's reads
@@ -647,6 +653,8 @@ namespace {
 std::atomic<long long> g_launches{0};
 }
 void count_launch() { g_launches.fetch_add(1); }       // for the library's other translation units
+int32_t* workspace_status_word(kap_workspace* ws) { return ws->d_status; }
+void workspace_lists_rewritten(kap_workspace* ws) { ws->plain_next = 1; }
 namespace {
 
 std::atomic<int> g_use_pdl{1};
@@ -735,13 +743,17 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     AttnParams p = p_in;
     p.cluster = ws->cluster_size;
     p.ring_slots = ws->ring_slots;
-    p.early_kv = (g_use_pdl.load() && g_early_kv.load()) ? 1 : 0;
+    // after the page lists were rewritten on the device, the prologue (which reads them ahead of
+    // the dependency wait) must not overlap the writer: one ordinary launch, then back to normal
+    const bool use_pdl = g_use_pdl.load() && !ws->plain_next;
+    ws->plain_next = 0;
+    p.early_kv = (use_pdl && g_early_kv.load()) ? 1 : 0;
 #ifdef KAP_TRACE
     p.trace = (g_trace && g_trace_next < g_trace_cap) ? g_trace + (size_t)(g_trace_next++) * 8192 * 8 : nullptr;
 #endif
     cudaLaunchAttribute attr[2];
     int n_attr = 0;
-    if (g_use_pdl.load()) {
+    if (use_pdl) {
         attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
         ++n_attr;

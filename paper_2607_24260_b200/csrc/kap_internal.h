@@ -51,6 +51,8 @@ struct kap_workspace {
     int32_t batch = 0, n_items = 0, n_groups = 0, n_merge_groups = 0, max_chunk = 0;
     int32_t ctas_per_wave = 0, row_tiles = 1, num_q_heads = 0, num_kv_heads = 0;
     int32_t has_nq = 0;            // schedule was made with an n_q array (verification path)
+    int32_t plain_next = 0;        // the page lists were just rewritten on the device: launch the
+                                   // next attention kernel as an ordinary (fully ordered) one
     int64_t total_rows = 0;        // sum over sequences of n_q
     // host (pinned) staging and device copies
     kap::WorkItem* h_items = nullptr;

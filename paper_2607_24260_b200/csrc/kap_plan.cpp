@@ -60,6 +60,35 @@ void splice(std::vector<Interval>& u, int32_t lo, int32_t hi) {
 
 struct Candidate { float score; int32_t lo, hi, index; };
 
+// pages touched by sorted disjoint intervals, ascending and unique; appended to `out` when given
+int32_t pages_of(const std::vector<Interval>& iv, int32_t page_size, std::vector<int32_t>* out) {
+    int32_t last_page = -1, n = 0;
+    for (const auto& x : iv) {
+        const int32_t p0 = std::max(last_page + 1, x.lo / page_size);
+        const int32_t p1 = (x.hi - 1) / page_size;
+        for (int32_t p = p0; p <= p1; ++p) { if (out) out->push_back(p); ++n; }
+        last_page = std::max(last_page, p1);
+    }
+    return n;
+}
+
+// Growing plans (kap_compile_growing_plan): the emitted list is the part of the plan that does not
+// move with the context length (sink + selected spans, or the whole prefix for a full plan),
+// followed by reserved entries that kap_refresh_recent fills from the current length.
+struct GrowOpts {
+    int32_t max_growth;
+    int32_t* tail_desc;      // [batch][3] = reserved entries, window tokens, first token they may cover
+};
+
+kap_status compile_impl(
+    int32_t batch, int32_t page_size, const int32_t* ctx_len, const int32_t* span_indptr,
+    const int32_t* span_start, const int32_t* span_len, const float* span_score,
+    const int32_t* budget_tokens, const int32_t* n_sink, const int32_t* n_recent,
+    const uint8_t* force_full, float s_max, const int32_t* bt_indptr, const int32_t* bt_pages,
+    int64_t plan_capacity, int32_t* plan_indptr, int32_t* plan_logical_pages,
+    int32_t* plan_phys_pages, int32_t* plan_flags, int32_t* selected_tokens,
+    uint16_t* plan_token_masks, const GrowOpts* grow);
+
 }  // namespace
 }  // namespace kap
 
@@ -76,7 +105,45 @@ extern "C" kap_status kap_compile_plan(
     int32_t* plan_phys_pages, int32_t* plan_flags, int32_t* selected_tokens,
     uint16_t* plan_token_masks)
 {
+    return kap::compile_impl(batch, page_size, ctx_len, span_indptr, span_start, span_len, span_score,
+                             budget_tokens, n_sink, n_recent, force_full, s_max, bt_indptr, bt_pages,
+                             plan_capacity, plan_indptr, plan_logical_pages, plan_phys_pages,
+                             plan_flags, selected_tokens, plan_token_masks, nullptr);
+}
+
+extern "C" kap_status kap_compile_growing_plan(
+    int32_t batch, int32_t page_size, const int32_t* ctx_len, const int32_t* span_indptr,
+    const int32_t* span_start, const int32_t* span_len, const float* span_score,
+    const int32_t* budget_tokens, const int32_t* n_sink, const int32_t* n_recent,
+    const uint8_t* force_full, float s_max, const int32_t* bt_indptr, const int32_t* bt_pages,
+    int32_t max_growth, int64_t plan_capacity, int32_t* plan_indptr, int32_t* plan_logical_pages,
+    int32_t* plan_phys_pages, uint16_t* plan_token_masks, int32_t* plan_flags,
+    int32_t* selected_tokens, int32_t* tail_desc)
+{
     using namespace kap;
+    if (max_growth < 0) return fail(KAP_ERR_INVALID_ARG, "max_growth %d < 0", max_growth);
+    if (!plan_token_masks || !plan_phys_pages || (batch > 0 && !tail_desc))
+        return fail(KAP_ERR_INVALID_ARG, "a growing plan needs plan_phys_pages, plan_token_masks and tail_desc");
+    if (!bt_indptr) return fail(KAP_ERR_INVALID_ARG, "a growing plan needs a block table");
+    const GrowOpts grow{max_growth, tail_desc};
+    return compile_impl(batch, page_size, ctx_len, span_indptr, span_start, span_len, span_score,
+                        budget_tokens, n_sink, n_recent, force_full, s_max, bt_indptr, bt_pages,
+                        plan_capacity, plan_indptr, plan_logical_pages, plan_phys_pages, plan_flags,
+                        selected_tokens, plan_token_masks, &grow);
+}
+
+namespace kap {
+namespace {
+
+kap_status compile_impl(
+    int32_t batch, int32_t page_size, const int32_t* ctx_len, const int32_t* span_indptr,
+    const int32_t* span_start, const int32_t* span_len, const float* span_score,
+    const int32_t* budget_tokens, const int32_t* n_sink, const int32_t* n_recent,
+    const uint8_t* force_full, float s_max, const int32_t* bt_indptr, const int32_t* bt_pages,
+    int64_t plan_capacity, int32_t* plan_indptr, int32_t* plan_logical_pages,
+    int32_t* plan_phys_pages, int32_t* plan_flags, int32_t* selected_tokens,
+    uint16_t* plan_token_masks, const GrowOpts* grow)
+{
     if (batch < 0) return fail(KAP_ERR_INVALID_ARG, "batch %d < 0", batch);
     if (page_size <= 0) return fail(KAP_ERR_INVALID_ARG, "page_size %d <= 0", page_size);
     if (!plan_indptr || !plan_flags || (!plan_logical_pages && plan_capacity > 0))
@@ -121,19 +188,28 @@ extern "C" kap_status kap_compile_plan(
     std::vector<int32_t> indptr(batch + 1, 0), flags(batch, 0), used_tokens(batch, 0);
     std::vector<int32_t> logical;
     std::vector<uint16_t> masks;
-    std::vector<Interval> u;
+    std::vector<Interval> u, fixed;     // fixed: the part of u that does not move with the length
     std::vector<Candidate> cand;
+    std::vector<int32_t> tail(grow ? (size_t)batch * 3 : 0, 0);
     for (int32_t b = 0; b < batch; ++b) {
         const int32_t L = ctx_len[b];
         const int32_t n_pages = (int32_t)(((int64_t)L + page_size - 1) / page_size);
         u.clear();
+        fixed.clear();
         int64_t used = 0;
         int32_t fl = 0;
+        const int64_t window = std::max(n_recent[b], 1);                // the last token is mandatory
+        bool moves = false;               // would another length have changed the selection?
         if (force_full && force_full[b]) {
             u.push_back({0, L});
+            if (grow) fixed.push_back({0, L});
             used = L;
             fl |= KAP_PLAN_FULL;
         } else {
+            if (grow) {
+                splice(fixed, 0, std::min(n_sink[b], L));
+                moves = (int64_t)n_sink[b] > (int64_t)L - window;
+            }
             splice(u, 0, std::min(n_sink[b], L));
             splice(u, std::max<int64_t>(0, (int64_t)L - n_recent[b]), L);
             splice(u, L - 1, L);
@@ -146,6 +222,11 @@ extern "C" kap_status kap_compile_plan(
                     const int64_t lo = std::max<int64_t>(0, span_start[i]);
                     const int64_t hi = std::min<int64_t>(L, (int64_t)span_start[i] + span_len[i]);
                     if (hi > lo) cand.push_back({span_score[i], (int32_t)lo, (int32_t)hi, i});
+                    // a span that reaches the recent window (or past the end) costs a different
+                    // number of tokens at another length
+                    if (grow && span_len[i] > 0 &&
+                        (int64_t)span_start[i] + span_len[i] > std::max<int64_t>(0, (int64_t)L - window))
+                        moves = true;
                 }
                 std::sort(cand.begin(), cand.end(), [](const Candidate& a, const Candidate& c) {
                     if (a.score != c.score) return a.score > c.score;
@@ -156,25 +237,22 @@ extern "C" kap_status kap_compile_plan(
                     const int64_t fresh = uncovered(u, c.lo, c.hi);
                     if (used + fresh <= budget_tokens[b]) {
                         splice(u, c.lo, c.hi);
+                        if (grow) splice(fixed, c.lo, c.hi);
                         used += fresh;
                     }
                 }
             }
         }
         // pages touched by the union, ascending and unique
-        int32_t last_page = -1, n_sel = 0;
-        for (const auto& iv : u) {
-            const int32_t p0 = std::max(last_page + 1, iv.lo / page_size);
-            const int32_t p1 = (iv.hi - 1) / page_size;
-            for (int32_t p = p0; p <= p1; ++p) { logical.push_back(p); ++n_sel; }
-            last_page = std::max(last_page, p1);
-        }
+        const int32_t n_sel = pages_of(u, page_size, grow ? nullptr : &logical);
+        const std::vector<Interval>& listed = grow ? fixed : u;
+        if (grow) pages_of(fixed, page_size, &logical);
         if (plan_token_masks) {
             // bit t of a listed page: token page*P + t lies in the union (intervals and pages both
             // ascend, so one forward sweep pairs them up)
             masks.resize(logical.size(), 0);
             size_t e = (size_t)indptr[b];
-            for (const auto& iv : u) {
+            for (const auto& iv : listed) {
                 while ((int64_t)logical[e] * page_size + page_size <= iv.lo) ++e;
                 for (size_t k = e; k < logical.size() && (int64_t)logical[k] * page_size < iv.hi; ++k) {
                     const int64_t base = (int64_t)logical[k] * page_size;
@@ -183,6 +261,23 @@ extern "C" kap_status kap_compile_plan(
                     masks[k] |= (uint16_t)(((1u << hi) - 1u) & ~((1u << lo) - 1u));
                 }
             }
+        }
+        if (grow) {
+            // reserved entries for the window [L' - window, L') at any later length L' (for a full
+            // plan: for every token from L on, up to max_growth of them); empty until refreshed
+            const bool full = (fl & KAP_PLAN_FULL) != 0;
+            int64_t reserve;
+            if (full)
+                reserve = grow->max_growth == 0 ? 0
+                        : ((int64_t)L + grow->max_growth - 1) / page_size - L / page_size + 1;
+            else
+                reserve = (window + page_size - 2) / page_size + 1;
+            for (int64_t r = 0; r < reserve; ++r) logical.push_back(0);
+            masks.resize(logical.size(), 0);
+            tail[(size_t)b * 3 + 0] = (int32_t)reserve;
+            tail[(size_t)b * 3 + 1] = full ? INT32_MAX : (int32_t)window;
+            tail[(size_t)b * 3 + 2] = full ? L : 0;
+            if (moves) fl |= KAP_PLAN_MOVES_WITH_LENGTH;
         }
         if ((double)n_sel / (double)n_pages > (double)s_max) fl |= KAP_PLAN_S_HIGH;
         if ((int64_t)logical.size() > (int64_t)INT32_MAX)
@@ -209,5 +304,9 @@ extern "C" kap_status kap_compile_plan(
         plan_flags[b] = flags[b];
         if (selected_tokens) selected_tokens[b] = used_tokens[b];
     }
+    if (grow && batch > 0) std::memcpy(grow->tail_desc, tail.data(), sizeof(int32_t) * tail.size());
     return KAP_OK;
 }
+
+}  // namespace
+}  // namespace kap

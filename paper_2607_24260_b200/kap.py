@@ -15,7 +15,7 @@ import numpy as np
 from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_DEVICE_INDEX = range(7)
-PLAN_FULL, PLAN_OVER_BUDGET, PLAN_S_HIGH = 1, 2, 4
+PLAN_FULL, PLAN_OVER_BUDGET, PLAN_S_HIGH, PLAN_MOVES_WITH_LENGTH = 1, 2, 4, 8
 
 _i32p, _f32p, _u8p, _vp = C.POINTER(C.c_int32), C.POINTER(C.c_float), C.POINTER(C.c_uint8), C.c_void_p
 
@@ -24,6 +24,12 @@ SIGNATURES = {
     "kap_compile_plan": (C.c_int, [C.c_int32, C.c_int32, _i32p, _i32p, _i32p, _i32p, _f32p, _i32p,
                                    _i32p, _i32p, _u8p, C.c_float, _i32p, _i32p, C.c_int64, _i32p,
                                    _i32p, _i32p, _i32p, _i32p, C.POINTER(C.c_uint16)]),
+    "kap_compile_growing_plan": (C.c_int, [C.c_int32, C.c_int32, _i32p, _i32p, _i32p, _i32p, _f32p,
+                                           _i32p, _i32p, _i32p, _u8p, C.c_float, _i32p, _i32p,
+                                           C.c_int32, C.c_int64, _i32p, _i32p, _i32p,
+                                           C.POINTER(C.c_uint16), _i32p, _i32p, _i32p]),
+    "kap_refresh_recent": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32,
+                                     C.c_int64, _vp, _vp, _vp]),
     "kap_workspace_create": (C.c_int, [C.POINTER(_vp), C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
     "kap_workspace_destroy": (None, [_vp]),
     "kap_schedule": (C.c_int, [_vp, C.c_int32, _i32p, _i32p, C.c_int32, C.c_int32, C.c_int32, _vp]),
@@ -140,6 +146,55 @@ def compile_plan(ctx_len, span_indptr, span_start, span_len, span_score, budget_
                 plan_phys_pages=None if phys is None else phys[:n].copy(), plan_flags=flags,
                 selected_tokens=sel,
                 plan_token_masks=None if masks is None else masks[:n].copy())
+
+
+def compile_growing_plan(ctx_len, span_indptr, span_start, span_len, span_score, budget_tokens,
+                         n_sink, n_recent, bt_indptr, bt_pages, force_full=None, s_max=1.0,
+                         page_size=16, max_growth=0, capacity=None):
+    """kap_compile_growing_plan on host arrays.  Returns the dict of compile_plan (lists = fixed
+    part + reserved entries) plus tail_desc int32 [B, 3]."""
+    ctx_len = _np(ctx_len, np.int32)
+    B = int(ctx_len.shape[0])
+    span_indptr, span_start = _np(span_indptr, np.int32), _np(span_start, np.int32)
+    span_len, span_score = _np(span_len, np.int32), _np(span_score, np.float32)
+    budget_tokens, n_sink = _np(budget_tokens, np.int32), _np(n_sink, np.int32)
+    n_recent, force_full = _np(n_recent, np.int32), _np(force_full, np.uint8)
+    bt_indptr, bt_pages = _np(bt_indptr, np.int32), _np(bt_pages, np.int32)
+    if capacity is None:
+        ps = max(page_size, 1)
+        capacity = int(sum((max(int(L), 0) + ps - 1) // ps + (max(int(r), 1) + ps - 2) // ps + 1
+                           + (max_growth + ps - 1) // ps + 1 for L, r in zip(ctx_len, n_recent)))
+    indptr = np.full(B + 1, -1, dtype=np.int32)
+    logical = np.full(max(1, capacity), -1, dtype=np.int32)
+    phys = np.full(max(1, capacity), -1, dtype=np.int32)
+    masks = np.zeros(max(1, capacity), dtype=np.uint16)
+    flags = np.full(B, -1, dtype=np.int32)
+    sel = np.full(B, -1, dtype=np.int32)
+    tail = np.full((B, 3), -1, dtype=np.int32)
+    _check(lib().kap_compile_growing_plan(
+        B, page_size, _ptr(ctx_len, C.c_int32), _ptr(span_indptr, C.c_int32),
+        _ptr(span_start, C.c_int32), _ptr(span_len, C.c_int32), _ptr(span_score, C.c_float),
+        _ptr(budget_tokens, C.c_int32), _ptr(n_sink, C.c_int32), _ptr(n_recent, C.c_int32),
+        _ptr(force_full, C.c_uint8), float(s_max), _ptr(bt_indptr, C.c_int32),
+        _ptr(bt_pages, C.c_int32), int(max_growth), int(capacity), _ptr(indptr, C.c_int32),
+        _ptr(logical, C.c_int32), _ptr(phys, C.c_int32), _ptr(masks, C.c_uint16),
+        _ptr(flags, C.c_int32), _ptr(sel, C.c_int32), _ptr(tail, C.c_int32)))
+    n = int(indptr[-1])
+    return dict(plan_indptr=indptr, plan_logical_pages=logical[:n].copy(),
+                plan_phys_pages=phys[:n].copy(), plan_flags=flags, selected_tokens=sel,
+                plan_token_masks=masks[:n].copy(), tail_desc=tail)
+
+
+def refresh_recent(plan_indptr, plan_logical_pages, plan_phys_pages, plan_token_masks, tail_desc,
+                   bt_indptr, bt_pages, ctx_len, num_pool_pages, ws: "Workspace | None" = None,
+                   device_status=None, page_size=16, stream=None):
+    """kap_refresh_recent on torch CUDA tensors (int32; masks as 16-bit words): rewrites the
+    reserved entries of a growing plan from the current device ctx_len."""
+    _check(lib().kap_refresh_recent(
+        _dptr(plan_indptr), _dptr(plan_logical_pages), _dptr(plan_phys_pages),
+        _dptr(plan_token_masks), _dptr(tail_desc), _dptr(bt_indptr), _dptr(bt_pages),
+        _dptr(ctx_len), int(ctx_len.shape[0]), int(page_size), int(num_pool_pages),
+        _dptr(device_status), None if ws is None else ws._h, _stream_ptr(stream)))
 
 
 def compile_workload(w, capacity=None):

@@ -290,6 +290,50 @@ def tiny_random(seed: int, batch: int = 3, max_len: int = 200, max_spans: int = 
                     num_pool_pages=pool, page_size=page_size)
 
 
+def growing_random(seed: int, batch: int = 4, max_doc: int = 600, growth: int = 40,
+                   max_spans: int = 10, overlap_every: int = 4) -> Workload:
+    """Sequences in the middle of generation: evidence spans lie in a document prefix
+    [0, L_doc), the context has already grown past it, and it will grow by up to ``growth`` more
+    tokens (the block tables already hold pages for them).  Most sequences have generated at least
+    n_recent tokens, so that spans and recent window are disjoint at every later length; every
+    ``overlap_every``-th one has not (its spans reach into the recent window).  Some sequences take
+    the full-context path."""
+    rng = rng_for(seed, "growing")
+    ctx, spans, budget, sink, recent, force, final = [], [], [], [], [], [], []
+    for b in range(batch):
+        L_doc = int(rng.integers(40, max_doc + 1))
+        n_recent = int(rng.integers(0, 40))
+        overlapping = overlap_every > 0 and b % overlap_every == overlap_every - 1
+        done = int(rng.integers(0, max(n_recent, 1))) if overlapping else \
+            max(n_recent, 1) + int(rng.integers(0, 50))
+        L = L_doc + done
+        n = int(rng.integers(0, max_spans + 1))
+        starts = rng.integers(0, L_doc, size=n)
+        lens = np.minimum(rng.integers(1, max(2, L_doc // 3), size=n), L_doc - starts)
+        scores = (rng.integers(0, 6, size=n) / 2.0).astype(np.float32)
+        if overlapping:                                   # one span over the document's tail
+            tail_len = min(L_doc, 24)
+            starts = np.append(starts, L_doc - tail_len)
+            lens = np.append(lens, tail_len)
+            scores = np.append(scores, np.float32(2.0))
+        spans.append((starts, lens, scores))
+        n_sink = int(rng.integers(0, 10))
+        sink.append(n_sink)
+        recent.append(n_recent)
+        budget.append(int(rng.integers(n_sink + n_recent, L_doc + n_recent + 8)))
+        force.append(int(rng.random() < 0.15))
+        ctx.append(L)
+        final.append(L + growth)
+    bi, bp, pool = block_tables(final, "shuffled", seed, "growing", PAGE_SIZE, 3)
+    si, ss, sl, sc = _pack_spans(spans)
+    i32 = lambda v: np.asarray(v, dtype=np.int32)
+    return Workload(name=f"growing{seed}", layers=1, ctx_len=i32(ctx), n_q=np.ones(batch, np.int32),
+                    span_indptr=si, span_start=ss, span_len=sl, span_score=sc,
+                    budget_tokens=i32(budget), n_sink=i32(sink), n_recent=i32(recent),
+                    force_full=np.asarray(force, dtype=np.uint8), bt_indptr=bi, bt_pages=bp,
+                    num_pool_pages=pool, note=f"growth={growth}")
+
+
 # ------------------------------------------------------------------------------------ value draws
 def host_qkv(w: Workload, seed: int, layer: int = 0, kv_std: float = 0.5, q_std: float = 1.0,
              q_rows: Optional[int] = None):
