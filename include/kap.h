@@ -327,7 +327,8 @@ kap_status kap_phase_model(double k, double h, double s, double w_main, double w
  * lists.  kap_selected_decode_attn on these arrays (plan_token_masks is required) then sees
  * exactly fixed part + window at the current length, and one kap_schedule (list lengths never
  * change) serves every step.  A page that holds both fixed and window tokens is listed twice with
- * disjoint masks; an entry with an empty mask is neither fetched nor computed.
+ * disjoint masks; a reserved entry that is not needed repeats the sequence's last page with an
+ * empty mask (read like any page, contributes nothing).
  *
  * A full-context plan (force_full) lists the whole prefix and reserves entries for every token
  * from ctx_len on, up to max_growth more tokens; for other sequences max_growth is not needed.
@@ -349,7 +350,8 @@ kap_status kap_phase_model(double k, double h, double s, double w_main, double w
  * like the attention calls.  Problems found on the device (a window page without a block-table
  * entry, a page outside the pool, a context that outgrew the reservation, ctx_len <= 0) set
  * 1 << KAP_ERR_DEVICE_INDEX in *device_status, or in the status word of `ws` when device_status is
- * NULL, and leave the affected entries empty.  `ws` (may be NULL) is the workspace of the
+ * NULL, and leave the affected entries empty (unchanged when the page of the last token itself
+ * is missing).  `ws` (may be NULL) is the workspace of the
  * attention call that will read the arrays: its next launch is then issued without programmatic
  * dependent launch, because the attention prologue reads the lists ahead of the dependency wait.
  * Errors: KAP_ERR_UNSUPPORTED (page_size > 16), KAP_ERR_INVALID_ARG, KAP_ERR_CUDA.

@@ -45,17 +45,28 @@ constexpr int kDefaultSlots = 8;                          // 8 slots -> 3 CTAs/S
 constexpr int kHalfTileBytes = kPageSize * 128;           // 16 tokens x 64 bf16 = 2048 B
 constexpr int kTileBytes = 2 * kHalfTileBytes;            // K (or V) of one page and head: 4096 B
 constexpr int kPageHeadBytes = 2 * kTileBytes;            // K + V: 8192 B
-constexpr int kMaxIds = 640;                              // page ids a CTA can hold (dynamic sharing up to this)
+constexpr int kMaxIds = 640;                              // page ids a CTA can hold (its own share of an item)
 constexpr int kScratchStride = kHeadDim + 8;              // floats per scratch row (bank spread)
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;         // per-CTA deadline for all waits
 
+// Page ids of a CTA: phys[cap], logical[cap], mask[cap] packed into one array, cap = kMaxIds.  A
+// cluster whose CTAs hold at most kPushIds ids and at most kPushRows query rows uses cap = kPushIds
+// and the rest of the array as the landing zone of the push-style cluster reduction (see the
+// epilogue): C * ceil(cells / C) <= kPushCells + 16 cells of (float4 o, float2 (m, l)) each.
+constexpr int kPushIds = 256;
+constexpr int kPushRows = 4;
+constexpr int kPushCells = kPushRows * 32;                // (row, 4-column) cells of the item
+constexpr int kZoneCells = kPushCells + kMaxCluster;
+constexpr int kIdBytes = kMaxIds * 10;
+constexpr int kZoneOff = kPushIds * 10;                   // byte offset of the landing zone
+static_assert(kZoneOff % 16 == 0 && kZoneOff + kZoneCells * 24 <= kIdBytes, "landing zone must fit behind the ids");
+
 struct SmemTail {                                         // control block in front of the ring
-    int32_t phys[kMaxIds];
-    int32_t logical[kMaxIds];
-    uint16_t mask[kMaxIds];                   // token-visibility bits of each page (all ones: whole page)
+    alignas(16) unsigned char ids[kIdBytes];  // phys, logical (int32) and token masks (uint16)
     int32_t slot_page[kMaxSlots];             // list index of the page in each ring slot, -1 = no more
     uint32_t slot_done[kMaxSlots];            // warps that have finished with the slot's current page
     unsigned long long full[kMaxSlots];
+    unsigned long long zone_full;             // completes when every peer has pushed its cells
     float m[kWarps][kRowTile];
     float l[kWarps][kRowTile];
     float cta_m[kRowTile * kMaxRowTiles];     // CTA-level state read by cluster peers
@@ -182,6 +193,41 @@ __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v 
 __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void cluster_arrive() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_dsmem_f32x4(uint32_t addr, float4 v) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_dsmem_f32x2(uint32_t addr, float a, float b) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
+// arrive on a peer's mbarrier; orders this thread's earlier remote stores before it (cluster scope)
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// bounded like mbar_wait, for a barrier that peers of the cluster arrive on
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint64_t deadline,
+                                                  volatile int32_t* timed_out) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((spin & 255u) == 0 && global_ns() > deadline) { *timed_out = 1; return false; }
+    }
+}
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta_rank) {
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
@@ -262,6 +308,11 @@ __device__ __forceinline__ void merge_group_cell(const AttnParams& p, const Merg
 // belongs to group i mod (4/RT) and is consumed by that group's RT warps (one per row tile).  Each
 // group owns 8/(4/RT) slots as a private ring; lane 0 of the group's first warp refills a slot as
 // soon as all RT warps have released it, so every group always has its whole ring in flight.
+//
+// kPush selects the cluster reduction: false = every CTA reads its peers' shared memory between two
+// cluster barriers; true = every CTA pushes its cells into the owners' landing zones (few rows and
+// short lists only: the host picks it when every item of the launch qualifies).
+template <bool kPush>
 __global__ void __launch_bounds__(kThreads, 3)
 kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
 {
@@ -278,35 +329,54 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
 
     // ---- prologue on static metadata only (work list, page lists, q_indptr): with programmatic
     // dependent launch it overlaps the tail of the previous kernel on the stream.
-    // A work item belongs to a cluster of C CTAs (C = 1: no cluster).  Its pages are dealt
-    // round-robin to the warp groups: over all groups of all C CTAs when the whole item's id list
-    // fits in shared memory, otherwise every CTA takes an even slice of the item and deals that.
+    // A work item belongs to a cluster of C CTAs (C = 1: no cluster).  CTA `rank` takes an even
+    // contiguous slice of the item's page list and stages only that; inside the slice the pages are
+    // dealt round-robin to the CTA's warp groups: the k-th page of group g is local id
+    // k * n_groups + g.
     const int C = p.cluster, rank = blockIdx.x % C;
-    WorkItem item = p.items[blockIdx.x / C];
-    const bool shared_list = (item.page_end - item.page_begin) <= kMaxIds;
-    if (!shared_list) {
-        const int n = item.page_end - item.page_begin, base = n / C, rem = n % C;
-        item.page_begin += rank * base + min(rank, rem);
-        item.page_end = item.page_begin + base + (rank < rem ? 1 : 0);
-    }
-    if (tid == 0 && item.page_end - item.page_begin > kMaxIds) atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX);
-    const int n_pages = min(item.page_end - item.page_begin, kMaxIds);   // the scheduler caps slices at 512
+    const WorkItem item = p.items[blockIdx.x / C];
     const int rows = item.n_q * p.G;                         // valid query rows of this item
     int RT = (rows + kRowTile - 1) / kRowTile;               // row tiles: 1, 2 or 4
     if (RT == 3) RT = 4;
+    const int n_groups = kWarps / RT;                        // warp groups
+    const int n_item = item.page_end - item.page_begin;      // pages of the whole item
+    const int slice0 = rank * (n_item / C) + min(rank, n_item % C);
+    int n_local = n_item / C + (rank < n_item % C ? 1 : 0);  // pages of this CTA
+    constexpr int kIdCap = kPush ? kPushIds : kMaxIds;
+    if (n_local > kIdCap) {                                  // the scheduler caps a CTA's share at 512
+        if (tid == 0) atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX);
+        n_local = kIdCap;
+    }
+    constexpr bool push = kPush;
+    constexpr int cap = push ? kPushIds : kMaxIds;
+    if (push && (C < 2 || rows > kPushRows)) {               // the host never launches this; the
+        if (tid == 0) atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX);   // landing zone would not fit
+        return;                                              // (same decision in the whole cluster)
+    }
+    int32_t* const id_phys = reinterpret_cast<int32_t*>(tail->ids);
+    int32_t* const id_logical = id_phys + cap;
+    uint16_t* const id_mask = reinterpret_cast<uint16_t*>(id_phys + 2 * cap);
+    const int n_cells = rows * 32;                           // (row, 4-column) cells of the item
+    const int per_rank = (n_cells + C - 1) / C;              // cells whose final merge a CTA owns
+    const int my_cells = max(0, min(n_cells, (rank + 1) * per_rank) - rank * per_rank);
     if (tid == 0) {
         for (int s = 0; s < n_slots; ++s) {
             mbar_init(smem_u32(&tail->full[s]), 1);
             tail->slot_done[s] = 0;
         }
+        if (push) mbar_init(smem_u32(&tail->zone_full), (uint32_t)max(1, my_cells * C));
         tail->timed_out = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map) : "memory");
     }
+    // first half of a cluster barrier; its second half sits in front of the pushes, where it
+    // guarantees that every peer has initialised its landing zone's barrier
+    if (push) cluster_arrive();
     const int64_t list0 = (int64_t)p.list_indptr[item.seq] + item.page_begin;
     const int64_t list_end = p.list_indptr[item.seq + 1];
     const int64_t q_row0 = p.q_indptr ? p.q_indptr[item.seq] : item.seq;
-    for (int i = tid; i < n_pages; i += kThreads) {
+    for (int j = tid; j < n_local; j += kThreads) {
+        const int i = slice0 + j;                            // entry of the item
         int32_t ph = 0;
         bool ok = (list0 + i) < list_end;
         if (ok) {
@@ -314,14 +384,13 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             ok = ph >= 0 && ph < p.num_pool_pages;
         }
         if (!ok) { ph = 0; atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX); }
-        tail->phys[i] = ph;
-        tail->logical[i] = p.logical_pages && ok ? p.logical_pages[list0 + i] : item.page_begin + i;
-        tail->mask[i] = p.token_masks && ok ? p.token_masks[list0 + i] : (uint16_t)0xFFFFu;
+        id_phys[j] = ph;
+        id_logical[j] = p.logical_pages && ok ? p.logical_pages[list0 + i] : item.page_begin + i;
+        id_mask[j] = p.token_masks && ok ? p.token_masks[list0 + i] : (uint16_t)0xFFFFu;
     }
     __syncthreads();
     KAP_TRACE_POINT(blockIdx.x, 1);
 
-    const int n_groups = kWarps / RT;                        // warp groups
     const int depth = n_slots / n_groups;                    // ring slots per group
     const int grp = warp / RT, rt = warp % RT;
     const bool producer = (rt == 0) && (lane == 0);           // fills the group's ring at the start
@@ -329,20 +398,14 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     const int v_row_off = p.Hkv * kPageSize;
     uint64_t policy;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    // the k-th page of this warp group is list entry first_idx + k * idx_stride
-    const int idx_stride = (shared_list ? C : 1) * n_groups;
-    const int first_idx = (shared_list ? rank : 0) * n_groups + grp;
+    const int group_pages = (n_local - grp + n_groups - 1) / n_groups;   // pages of this warp group
     // put the group's k-th page into ring slot s, or publish "no more pages" there
     auto fill = [&](int s, int k) {
         const uint32_t bar = smem_u32(&tail->full[s]);
-        const int idx = first_idx + k * idx_stride;
-        if (idx < n_pages) {
+        const int idx = k * n_groups + grp;                  // local id
+        if (k < group_pages) {
             tail->slot_page[s] = idx;
-            if (tail->mask[idx] == 0) {                      // no visible token: nothing to fetch
-                mbar_arrive(bar);
-                return;
-            }
-            const int y = tail->phys[idx] * rows_per_page + item.kv_head * kPageSize;
+            const int y = id_phys[idx] * rows_per_page + item.kv_head * kPageSize;
             const uint32_t dst = smem_u32(ring + s * kPageHeadBytes);
             mbar_expect_tx(bar, kPageHeadBytes);
             tma_load_2d(dst, &kv_map, 0, y, bar, policy);
@@ -366,8 +429,8 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         if (producer) {
             const int fresh_from = L_hint - item.n_q;
             while (filled < depth) {
-                const int idx = first_idx + filled * idx_stride;
-                if (idx >= n_pages || tail->logical[idx] * kPageSize + kPageSize - 1 >= fresh_from) break;
+                const int idx = filled * n_groups + grp;
+                if (filled >= group_pages || id_logical[idx] * kPageSize + kPageSize - 1 >= fresh_from) break;
                 fill(grp * depth + filled, filled);
                 ++filled;
             }
@@ -431,85 +494,83 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         if (i == 0) KAP_TRACE_POINT(blockIdx.x, 3);
         const int page = tail->slot_page[s];
         if (page < 0 || tail->timed_out) break;              // the list is exhausted
-        const uint32_t tmask = tail->mask[page];
-        if (tmask != 0u) {                                   // a page without a visible token was not fetched
-            const uint32_t kb = smem_u32(ring + s * kPageHeadBytes);
-            const uint32_t vb = kb + kTileBytes;
-            const int tok0 = tail->logical[page] * kPageSize;
+        const uint32_t tmask = id_mask[page];
+        const uint32_t kb = smem_u32(ring + s * kPageHeadBytes);
+        const uint32_t vb = kb + kTileBytes;
+        const int tok0 = id_logical[page] * kPageSize;
 
-            // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
-            float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
+        float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                uint32_t b0, b1, b2, b3;
-                ldsm_x4(kb + (ks >> 2) * kHalfTileBytes + k_tok * 128
-                           + ((((ks & 3) * 2 + k_cbit) ^ lr) << 4), b0, b1, b2, b3);
-                mma_bf16(sacc[0], qf[ks], b0, b1);
-                mma_bf16(sacc[1], qf[ks], b2, b3);
-            }
-            if (tok0 + kPageSize - 1 > full_vis_limit || tmask != 0xFFFFu) {
-                // page reaches into the causal / tail region, or only some of its tokens are in the
-                // selected union: mask per element
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4(kb + (ks >> 2) * kHalfTileBytes + k_tok * 128
+                       + ((((ks & 3) * 2 + k_cbit) ^ lr) << 4), b0, b1, b2, b3);
+            mma_bf16(sacc[0], qf[ks], b0, b1);
+            mma_bf16(sacc[1], qf[ks], b2, b3);
+        }
+        if (tok0 + kPageSize - 1 > full_vis_limit || tmask != 0xFFFFu) {
+            // page reaches into the causal / tail region, or only some of its tokens are in the
+            // selected union: mask per element
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt)
+            for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int slot = nt * 8 + tid4 * 2 + (e & 1);
-                        if (tok0 + slot > pos_row[e >> 1] || !((tmask >> slot) & 1u)) sacc[nt][e] = -INFINITY;
-                    }
-                // value rows past the end of the context may hold anything (even NaN): zero them
-                const int first_bad = L - tok0;
-                if (first_bad < kPageSize) {
-                    if (lane < 16) {
-                        for (int r = max(first_bad, 0); r < kPageSize; ++r)
-                            *reinterpret_cast<uint4*>(ring + s * kPageHeadBytes + kTileBytes
-                                                      + (lane >> 3) * kHalfTileBytes + r * 128
-                                                      + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
+                for (int e = 0; e < 4; ++e) {
+                    const int slot = nt * 8 + tid4 * 2 + (e & 1);
+                    if (tok0 + slot > pos_row[e >> 1] || !((tmask >> slot) & 1u)) sacc[nt][e] = -INFINITY;
                 }
-            }
-            // online softmax (base 2): rows gid (e = 0,1) and gid + 8 (e = 2,3)
-            float mx[2];
-            mx[0] = fmaxf(fmaxf(sacc[0][0], sacc[0][1]), fmaxf(sacc[1][0], sacc[1][1]));
-            mx[1] = fmaxf(fmaxf(sacc[0][2], sacc[0][3]), fmaxf(sacc[1][2], sacc[1][3]));
-            float corr[2], mu[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
-                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-                const float mn = fmaxf(m_run[h], mx[h] * sc);
-                mu[h] = (mn == -INFINITY) ? 0.f : mn;
-                corr[h] = ex2(m_run[h] - mu[h]);
-                m_run[h] = mn;
-            }
-            uint32_t pa[4];      // P as the A operand of P V (rows gid / gid+8, tokens 0-7 / 8-15)
-            pa[0] = pack_bf16(ex2(fmaf(sacc[0][0], sc, -mu[0])), ex2(fmaf(sacc[0][1], sc, -mu[0])));
-            pa[1] = pack_bf16(ex2(fmaf(sacc[0][2], sc, -mu[1])), ex2(fmaf(sacc[0][3], sc, -mu[1])));
-            pa[2] = pack_bf16(ex2(fmaf(sacc[1][0], sc, -mu[0])), ex2(fmaf(sacc[1][1], sc, -mu[0])));
-            pa[3] = pack_bf16(ex2(fmaf(sacc[1][2], sc, -mu[1])), ex2(fmaf(sacc[1][3], sc, -mu[1])));
-            // the row sums use the rounded weights, so out = sum(p v) / sum(p) is a true average
-            l_run[0] = fmaf(l_run[0], corr[0],
-                            (bf16_lo(pa[0]) + bf16_hi(pa[0])) + (bf16_lo(pa[2]) + bf16_hi(pa[2])));
-            l_run[1] = fmaf(l_run[1], corr[1],
-                            (bf16_lo(pa[1]) + bf16_hi(pa[1])) + (bf16_lo(pa[3]) + bf16_hi(pa[3])));
-            if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
-#pragma unroll
-                for (int n = 0; n < 16; ++n) {
-                    o[n][0] *= corr[0]; o[n][1] *= corr[0];
-                    o[n][2] *= corr[1]; o[n][3] *= corr[1];
+            // value rows past the end of the context may hold anything (even NaN): zero them
+            const int first_bad = L - tok0;
+            if (first_bad < kPageSize) {
+                if (lane < 16) {
+                    for (int r = max(first_bad, 0); r < kPageSize; ++r)
+                        *reinterpret_cast<uint4*>(ring + s * kPageHeadBytes + kTileBytes
+                                                  + (lane >> 3) * kHalfTileBytes + r * 128
+                                                  + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
             }
-            // O += P V   (16 n-tiles of 8 output columns, two per ldmatrix)
+        }
+        // online softmax (base 2): rows gid (e = 0,1) and gid + 8 (e = 2,3)
+        float mx[2];
+        mx[0] = fmaxf(fmaxf(sacc[0][0], sacc[0][1]), fmaxf(sacc[1][0], sacc[1][1]));
+        mx[1] = fmaxf(fmaxf(sacc[0][2], sacc[0][3]), fmaxf(sacc[1][2], sacc[1][3]));
+        float corr[2], mu[2];
 #pragma unroll
-            for (int n2 = 0; n2 < 8; ++n2) {
-                uint32_t v0, v1, v2, v3;
-                ldsm_x4_t(vb + (n2 >> 2) * kHalfTileBytes + v_tok * 128
-                             + ((((n2 & 3) * 2 + v_cbit) ^ lr) << 4), v0, v1, v2, v3);
-                mma_bf16(o[2 * n2], pa, v0, v1);
-                mma_bf16(o[2 * n2 + 1], pa, v2, v3);
+        for (int h = 0; h < 2; ++h) {
+            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+            const float mn = fmaxf(m_run[h], mx[h] * sc);
+            mu[h] = (mn == -INFINITY) ? 0.f : mn;
+            corr[h] = ex2(m_run[h] - mu[h]);
+            m_run[h] = mn;
+        }
+        uint32_t pa[4];      // P as the A operand of P V (rows gid / gid+8, tokens 0-7 / 8-15)
+        pa[0] = pack_bf16(ex2(fmaf(sacc[0][0], sc, -mu[0])), ex2(fmaf(sacc[0][1], sc, -mu[0])));
+        pa[1] = pack_bf16(ex2(fmaf(sacc[0][2], sc, -mu[1])), ex2(fmaf(sacc[0][3], sc, -mu[1])));
+        pa[2] = pack_bf16(ex2(fmaf(sacc[1][0], sc, -mu[0])), ex2(fmaf(sacc[1][1], sc, -mu[0])));
+        pa[3] = pack_bf16(ex2(fmaf(sacc[1][2], sc, -mu[1])), ex2(fmaf(sacc[1][3], sc, -mu[1])));
+        // the row sums use the rounded weights, so out = sum(p v) / sum(p) is a true average
+        l_run[0] = fmaf(l_run[0], corr[0],
+                        (bf16_lo(pa[0]) + bf16_hi(pa[0])) + (bf16_lo(pa[2]) + bf16_hi(pa[2])));
+        l_run[1] = fmaf(l_run[1], corr[1],
+                        (bf16_lo(pa[1]) + bf16_hi(pa[1])) + (bf16_lo(pa[3]) + bf16_hi(pa[3])));
+        if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+            for (int n = 0; n < 16; ++n) {
+                o[n][0] *= corr[0]; o[n][1] *= corr[0];
+                o[n][2] *= corr[1]; o[n][3] *= corr[1];
             }
+        }
+        // O += P V   (16 n-tiles of 8 output columns, two per ldmatrix)
+#pragma unroll
+        for (int n2 = 0; n2 < 8; ++n2) {
+            uint32_t v0, v1, v2, v3;
+            ldsm_x4_t(vb + (n2 >> 2) * kHalfTileBytes + v_tok * 128
+                         + ((((n2 & 3) * 2 + v_cbit) ^ lr) << 4), v0, v1, v2, v3);
+            mma_bf16(o[2 * n2], pa, v0, v1);
+            mma_bf16(o[2 * n2 + 1], pa, v2, v3);
         }
         // Done with the slot.  The last of the group's RT warps to get here refills it with the
         // group's page i + depth; nobody waits for anybody.  The fences order this warp's reads
@@ -559,6 +620,7 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     // Combine the warp groups: the CTA-level state of row R ends up in scratch row R (the region
     // of warp R / 16 of group 0, which only this cell's thread reads) and cta_m[R], cta_l[R]; with
     // one CTA per item it goes straight to global memory instead.
+    if (push) cluster_wait();                          // every peer's landing zone is ready
     for (int idx = tid; idx < rows * 32; idx += kThreads) {
         const int R = idx >> 5, c4 = idx & 31;
         const int t = R / kRowTile, r = R % kRowTile;
@@ -576,19 +638,51 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
                 *(reinterpret_cast<float4*>(p.part_o + prow * kHeadDim) + c4) = res.o;
                 if (c4 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(res.m, res.l);
             }
+        } else if (push) {
+            // Push-style cluster reduction: the cell goes straight into the landing zone of the
+            // CTA that owns it (slot: this CTA's rank), followed by an arrive on the owner's
+            // barrier that orders the stores before it.  Nobody reads this CTA's shared memory, so
+            // it may exit as soon as its own cells are complete.
+            const int owner = idx / per_rank, slot = rank * per_rank + idx % per_rank;
+            unsigned char* zone = tail->ids + kZoneOff;
+            st_dsmem_f32x4(map_to_cta(smem_u32(zone + slot * 16), owner), res.o);
+            st_dsmem_f32x2(map_to_cta(smem_u32(zone + kZoneCells * 16 + slot * 8), owner), res.m, res.l);
+            mbar_arrive_remote(map_to_cta(smem_u32(&tail->zone_full), owner));
         } else {
             *reinterpret_cast<float4*>(all + R * kScratchStride + c4 * 4) = res.o;
             if (c4 == 0) { m_flat[R] = res.m; l_flat[R] = res.l; }
         }
     }
-    if (C > 1) {
+    if (push) {
+        // owner side: cell `tid` of this CTA's share is complete once all C CTAs have pushed
+        if (tid < my_cells) {
+            if (mbar_wait_cluster(smem_u32(&tail->zone_full), 0, deadline, &tail->timed_out)) {
+                const int idx = rank * per_rank + tid;
+                const int R = idx >> 5, c4 = idx & 31;
+                const unsigned char* zone = tail->ids + kZoneOff;
+                Merged res; res.m = -INFINITY; res.l = 0.f; res.o = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int u = 0; u < C; ++u) {
+                    const int slot = u * per_rank + tid;
+                    const float2 ml = *reinterpret_cast<const float2*>(zone + kZoneCells * 16 + slot * 8);
+                    merge_into(res, ml.x, ml.y, *reinterpret_cast<const float4*>(zone + slot * 16));
+                }
+                if (single) {
+                    store_final(p, q_row0 + R / p.G, item.kv_head * p.G + R % p.G, c4, res);
+                } else {
+                    const int64_t prow = (int64_t)item.split * p.rows_cap + R;
+                    *(reinterpret_cast<float4*>(p.part_o + prow * kHeadDim) + c4) = res.o;
+                    if (c4 == 0) *reinterpret_cast<float2*>(p.part_ml + prow * 2) = make_float2(res.m, res.l);
+                }
+            } else {
+                atomicOr(p.status, 1 << KAP_ERR_TIMEOUT);
+            }
+        }
+    } else if (C > 1) {
         // Cluster reduction through distributed shared memory: after the first cluster barrier
         // every CTA's state is visible to its peers; rank r merges its share of the (row, column)
         // cells over all C CTAs and writes them out; the second barrier keeps every CTA's shared
         // memory alive until all peers have read it.
         cluster_sync();
-        const int n_cells = rows * 32;
-        const int per_rank = (n_cells + C - 1) / C;
         const int c_end = min(n_cells, (rank + 1) * per_rank);
         for (int idx = rank * per_rank + tid; idx < c_end; idx += kThreads) {
             const int R = idx >> 5, c4 = idx & 31;
@@ -732,10 +826,14 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     if (st != KAP_OK) return st;
     // function attributes are per device: set them once for the workspace's device
     if (!ws->attrs_set) {
-        cudaError_t ae = cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t ae = cudaFuncSetAttribute(kap_attn_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               smem_bytes_for(kMaxSlots));
+        if (ae == cudaSuccess)
+            ae = cudaFuncSetAttribute(kap_attn_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      smem_bytes_for(kMaxSlots));
         if (ae != cudaSuccess) return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ae));
-        cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        cudaFuncSetAttribute(kap_attn_split_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        cudaFuncSetAttribute(kap_attn_split_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         cudaGetLastError();
         ws->attrs_set = 1;
     }
@@ -773,7 +871,10 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel, *map, p));
+    // few rows and short lists in every item (the proposal path): push-style cluster reduction
+    const bool push = ws->cluster_size > 1 && ws->max_nq * p.G <= kPushRows && ws->max_chunk <= kPushIds;
+    if (push) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<true>, *map, p));
+    else KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<false>, *map, p));
     g_launches.fetch_add(1);
     if (ws->n_merge_groups > 0) {
         const int rows = ws->max_nq * p.G;
@@ -888,10 +989,10 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     KAP_CUDA(cudaSetDevice(ws->device));
     const int ring_slots = g_ring_slots.load();
     const int smem = smem_bytes_for(ring_slots);
-    cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(kap_attn_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          smem_bytes_for(kMaxSlots));
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel, kThreads, smem) != cudaSuccess || occ < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel<false>, kThreads, smem) != cudaSuccess || occ < 1)
         occ = 1;
     const int want = g_ctas_per_sm.load();
     const int per_sm = want > 0 ? std::min(want, occ) : occ;
@@ -899,7 +1000,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     ws->ring_slots = ring_slots;
     ws->ctas_per_wave = per_sm * ws->sm_count;
     int32_t slots[kMaxCluster] = {ws->ctas_per_wave};
-    cudaFuncSetAttribute(kap_attn_split_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    cudaFuncSetAttribute(kap_attn_split_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     cudaGetLastError();
     for (int c = 2; c <= kMaxCluster; ++c) {
         if (c > g_max_cluster.load()) continue;
@@ -912,7 +1013,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         cc.dynamicSmemBytes = smem;
         cc.attrs = ca; cc.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
+        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel<false>, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
         slots[c - 1] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
     }
     // a one-wave schedule leaves a third of the SM's CTA slots to the next kernel's early CTAs
@@ -1161,7 +1262,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
         if (!g_static_ready[dev]) {
             void* ptr = nullptr;
             KAP_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
-            KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel,
+            KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel<false>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           smem_bytes_for(kMaxSlots)));
             g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
@@ -1216,7 +1317,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
     g_launches.fetch_add(1);
     // plain launches: the work list was written by the kernel just before, so the split kernel
     // must not start early
-    kap_attn_split_kernel<<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
+    kap_attn_split_kernel<false><<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
     KAP_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     if (num_splits > 1) {

@@ -5,8 +5,8 @@
 // sequence.  This kernel rewrites the reserved entries from the current device-side ctx_len: the
 // pages of the recent window [L - n_recent, L) (Section 3.2: each proposal step sees the tokens
 // written before it), with a 16-bit token mask that leaves out the tokens the fixed part already
-// holds, so that no token is counted twice.  Unused reserved entries get an empty mask; the
-// attention kernel neither fetches nor computes such an entry.
+// holds, so that no token is counted twice.  Unused reserved entries repeat the sequence's last
+// page with an empty mask: the attention kernel reads it like any page and it contributes nothing.
 #include <cuda_runtime.h>
 
 #include "kap_internal.h"
@@ -45,8 +45,16 @@ kap_refresh_recent_kernel(const int32_t* __restrict__ plan_indptr, int32_t* plan
     if (needed > reserved && threadIdx.x == 0 && status)   // the context outgrew the reservation
         atomicOr(status, 1 << KAP_ERR_DEVICE_INDEX);
     const int n_bt = bt_indptr[b + 1] - bt_indptr[b];
+    // an entry that lists nothing still names a page the kernel will read: the last page of the
+    // context (its rows below the length hold real tokens, the kernel zeroes the rest)
+    const long long last_page = (L - 1) / page_size;
+    const int32_t idle_phys = last_page < n_bt ? bt_pages[bt_indptr[b] + last_page] : -1;
+    if (idle_phys < 0 || idle_phys >= num_pool_pages) {
+        if (threadIdx.x == 0 && status) atomicOr(status, 1 << KAP_ERR_DEVICE_INDEX);
+        return;                                            // entries keep their previous contents
+    }
     for (int r = threadIdx.x; r < reserved; r += blockDim.x) {
-        int32_t logical = 0, phys = 0;
+        int32_t logical = (int32_t)last_page, phys = idle_phys;
         uint32_t bits = 0;
         if (r < needed) {
             const long long p = first_page + r;

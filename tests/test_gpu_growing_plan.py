@@ -143,6 +143,8 @@ def test_growth_loop_in_one_graph(seed, steps):
 def test_refresh_reports_outgrown_reservation_and_missing_pages():
     w = synth.growing_random(5, batch=3, growth=64, overlap_every=0)
     w.force_full[:] = [1, 0, 0]
+    w.n_recent[2] = 30
+    w.ctx_len[2] = max(int(w.ctx_len[2]), 64)
     g = _grow(w, 8)                                         # the full plan may grow by 8 tokens only
     _, pool_bits = synth.host_qkv(w, 5, q_rows=3)
     dev = _Device(w, g, pool_bits)
@@ -157,16 +159,26 @@ def test_refresh_reports_outgrown_reservation_and_missing_pages():
     with pytest.raises(kap.KapError) as e:
         dev.ws.check()
     assert e.value.code == kap.ERR_DEVICE_INDEX
-    # a window page the block table does not hold
+    # a window page without a valid block-table entry: reported, that entry stays empty
     dev.ctx.copy_(gu.i32(w.ctx_len))
-    short = w.bt_indptr.copy()
-    short[3] = short[2] + int(w.ctx_len[2] - 1) // P        # seq 2 loses the page of its last token
-    short = gu.i32(short)
+    L2 = int(w.ctx_len[2])
+    first_window_page = (L2 - 30) // P                      # n_recent[2] = 30: the window spans >= 2 pages
+    assert first_window_page < (L2 - 1) // P
+    holes = w.bt_pages.copy()
+    holes[w.bt_indptr[2] + first_window_page] = -1
     status = torch.zeros(1, dtype=torch.int32, device=gu.DEV)
-    kap.refresh_recent(dev.indptr, dev.logical, dev.phys, dev.masks, dev.tail, short, dev.bt_pages,
+    kap.refresh_recent(dev.indptr, dev.logical, dev.phys, dev.masks, dev.tail, dev.bt_indptr, gu.i32(holes),
                        dev.ctx, dev.n_pool, device_status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 1 << kap.ERR_DEVICE_INDEX
     lst = dev.listed_tokens(2)
-    assert (int(w.ctx_len[2]) - 1) not in lst               # the affected entry stays empty
+    assert (L2 - 1) in lst and not any(t // P == first_window_page and t >= L2 - 30 for t in lst)
+    # the page of the last token itself is missing: reported
+    short = w.bt_indptr.copy()
+    short[3] = short[2] + (L2 - 1) // P
+    status.zero_()
+    kap.refresh_recent(dev.indptr, dev.logical, dev.phys, dev.masks, dev.tail, gu.i32(short), dev.bt_pages,
+                       dev.ctx, dev.n_pool, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1 << kap.ERR_DEVICE_INDEX
     dev.ws.close()
