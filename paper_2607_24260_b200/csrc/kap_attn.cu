@@ -97,6 +97,7 @@ struct AttnParams {
     int32_t* status;
     long long num_pool_pages;
     int32_t Hq, Hkv, G, rows_cap;
+    int32_t batch;                   // sequences (entries of list_indptr / q_indptr minus one)
     int32_t cluster, early_kv;       // CTAs per work item (cluster size); early KV prefetch
     int32_t ring_slots;              // page slots in the shared-memory ring (8, 12, 16 or 24)
     float scale_log2;                // sm_scale * log2(e)
@@ -333,8 +334,18 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     // contiguous slice of the item's page list and stages only that; inside the slice the pages are
     // dealt round-robin to the CTA's warp groups: the k-th page of group g is local id
     // k * n_groups + g.
+    // The prologue's global loads form a chain (work item -> list offsets -> page ids); under a
+    // saturated memory system each link costs ~0.5 us, so the chain is kept to two links: the
+    // offset arrays of the whole batch are copied to shared memory (the ring is still unused)
+    // alongside the work-item load instead of after it.
     const int C = p.cluster, rank = blockIdx.x % C;
     const WorkItem item = p.items[blockIdx.x / C];
+    int32_t* const offs = reinterpret_cast<int32_t*>(ring);  // [batch + 1] list offsets, then q offsets
+    for (int t = tid; t <= p.batch; t += kThreads) {
+        offs[t] = p.list_indptr[t];
+        if (p.q_indptr) offs[p.batch + 1 + t] = p.q_indptr[t];
+    }
+    __syncthreads();
     const int rows = item.n_q * p.G;                         // valid query rows of this item
     int RT = (rows + kRowTile - 1) / kRowTile;               // row tiles: 1, 2 or 4
     if (RT == 3) RT = 4;
@@ -372,23 +383,25 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     // first half of a cluster barrier; its second half sits in front of the pushes, where it
     // guarantees that every peer has initialised its landing zone's barrier
     if (push) cluster_arrive();
-    const int64_t list0 = (int64_t)p.list_indptr[item.seq] + item.page_begin;
-    const int64_t list_end = p.list_indptr[item.seq + 1];
-    const int64_t q_row0 = p.q_indptr ? p.q_indptr[item.seq] : item.seq;
+    const int64_t list0 = (int64_t)offs[item.seq] + item.page_begin;
+    const int64_t list_end = offs[item.seq + 1];
+    const int64_t q_row0 = p.q_indptr ? offs[p.batch + 1 + item.seq] : item.seq;
     for (int j = tid; j < n_local; j += kThreads) {
         const int i = slice0 + j;                            // entry of the item
-        int32_t ph = 0;
-        bool ok = (list0 + i) < list_end;
-        if (ok) {
-            ph = p.phys_pages[list0 + i];
-            ok = ph >= 0 && ph < p.num_pool_pages;
-        }
-        if (!ok) { ph = 0; atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX); }
+        // the three loads are independent of one another: one round trip
+        const bool listed = (list0 + i) < list_end;
+        int32_t ph = listed ? p.phys_pages[list0 + i] : -1;
+        const int32_t lg = listed && p.logical_pages ? p.logical_pages[list0 + i] : item.page_begin + i;
+        const uint16_t mk = listed && p.token_masks ? p.token_masks[list0 + i] : (uint16_t)0xFFFFu;
+        if (ph < 0 || ph >= p.num_pool_pages) { ph = 0; atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX); }
         id_phys[j] = ph;
-        id_logical[j] = p.logical_pages && ok ? p.logical_pages[list0 + i] : item.page_begin + i;
-        id_mask[j] = p.token_masks && ok ? p.token_masks[list0 + i] : (uint16_t)0xFFFFu;
+        id_logical[j] = lg;
+        id_mask[j] = mk;
     }
     __syncthreads();
+    // the offsets in the ring were written by ordinary stores; the bulk copies that overwrite them
+    // next go through the asynchronous proxy
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     KAP_TRACE_POINT(blockIdx.x, 1);
 
     const int depth = n_slots / n_groups;                    // ring slots per group
@@ -1080,7 +1093,7 @@ static AttnParams base_params(kap_workspace* ws, int32_t hq, int32_t hkv, float 
     p.items = ws->d_items; p.groups = ws->d_groups; p.part_o = ws->d_part_o;
     p.part_ml = ws->d_part_ml; p.status = ws->d_status;
     p.num_pool_pages = num_pool_pages; p.Hq = hq; p.Hkv = hkv; p.G = hq / hkv;
-    p.rows_cap = ws->max_rows;
+    p.rows_cap = ws->max_rows; p.batch = ws->batch;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
     return p;
 }
@@ -1299,7 +1312,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
     p.out = (__nv_bfloat16*)out; p.lse = lse;
     p.status = reinterpret_cast<int32_t*>(base);
     p.num_pool_pages = num_pool_pages; p.Hq = num_q_heads; p.Hkv = num_kv_heads; p.G = rows;
-    p.rows_cap = rows; p.cluster = 1; p.early_kv = 0; p.ring_slots = kDefaultSlots;
+    p.rows_cap = rows; p.batch = batch; p.cluster = 1; p.early_kv = 0; p.ring_slots = kDefaultSlots;
     p.scale_log2 = sm_scale * 1.4426950408889634f;
 #ifdef KAP_TRACE
     p.trace = nullptr;
