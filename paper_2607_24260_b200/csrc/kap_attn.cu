@@ -380,8 +380,8 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map) : "memory");
     }
-    // first half of a cluster barrier; its second half sits in front of the pushes, where it
-    // guarantees that every peer has initialised its landing zone's barrier
+    // first half of a cluster barrier; its second half (before the main loop) guarantees that
+    // every peer has initialised its landing zone's barrier before anybody pushes
     if (push) cluster_arrive();
     const int64_t list0 = (int64_t)offs[item.seq] + item.page_begin;
     const int64_t list_end = offs[item.seq + 1];
@@ -472,6 +472,9 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         for (; filled < depth; ++filled) fill(grp * depth + filled, filled);
     const int L = p.ctx_len[item.seq];
     const uint64_t deadline = global_ns() + kWaitBudgetNs;
+    // second half of the prologue's cluster barrier: by now every peer has long arrived, so this
+    // costs nothing here, and the epilogue may push without any further synchronisation
+    if (push) cluster_wait();
 
     // Q fragments (A operand, 16 rows x 128) straight from global memory, zero for padding rows.
     uint32_t qf[8][4];
@@ -614,11 +617,13 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     __syncthreads();                                   // all tile reads done: the ring is scratch now
     float* scratch = reinterpret_cast<float*>(ring) + warp * (kRowTile * kScratchStride);
 #pragma unroll
-    for (int n = 0; n < 16; ++n) {
-        *reinterpret_cast<float2*>(scratch + gid * kScratchStride + n * 8 + tid4 * 2) =
-            make_float2(o[n][0], o[n][1]);
-        *reinterpret_cast<float2*>(scratch + (gid + 8) * kScratchStride + n * 8 + tid4 * 2) =
-            make_float2(o[n][2], o[n][3]);
+    for (int n = 0; n < 16; ++n) {                      // padding rows are never read back
+        if (rt * kRowTile + gid < rows)
+            *reinterpret_cast<float2*>(scratch + gid * kScratchStride + n * 8 + tid4 * 2) =
+                make_float2(o[n][0], o[n][1]);
+        if (rt * kRowTile + gid + 8 < rows)
+            *reinterpret_cast<float2*>(scratch + (gid + 8) * kScratchStride + n * 8 + tid4 * 2) =
+                make_float2(o[n][2], o[n][3]);
     }
     if (tid4 == 0) {
         tail->m[warp][gid] = m_run[0];     tail->l[warp][gid] = l_run[0];
@@ -633,7 +638,7 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     // Combine the warp groups: the CTA-level state of row R ends up in scratch row R (the region
     // of warp R / 16 of group 0, which only this cell's thread reads) and cta_m[R], cta_l[R]; with
     // one CTA per item it goes straight to global memory instead.
-    if (push) cluster_wait();                          // every peer's landing zone is ready
+    KAP_TRACE_POINT(blockIdx.x, 6);
     for (int idx = tid; idx < rows * 32; idx += kThreads) {
         const int R = idx >> 5, c4 = idx & 31;
         const int t = R / kRowTile, r = R % kRowTile;

@@ -31,11 +31,13 @@ int64_t chunks_for(const int32_t* len, int32_t batch, int32_t hkv, int64_t t) {
 // Cost model used to pick the cluster size and the number of waves, in units of "pages streamed
 // by one CTA": a CTA pays a fixed start-up / epilogue cost, a launch whose groups need more than
 // one cluster pays for the separate merge pass, a cluster pays for its two cluster barriers and
-// the looser placement of its CTAs (measured: about 1.6 pages per CTA of the cluster).
+// the looser placement of its CTAs (measured: about 1.6 pages per CTA of the cluster; half of
+// that when the kernel can use its push-style reduction, i.e. for items of at most 4 query rows).
 constexpr int64_t kFixedPages = 6;                        // + rows / 2: wider items start and end slower
 constexpr int64_t kMergePassPages = 9;
 constexpr int64_t kLaterWavePages = 40;
 constexpr int64_t kClusterPagesX5 = 8;                    // per CTA of a cluster, in fifths of a page
+constexpr int64_t kPushClusterPagesX5 = 4;                // same, when the kernel reduces by pushing (<= 4 rows)
 constexpr int32_t kDefaultChunkCap = 512;     // per CTA; also the size of the kernel's page-id buffer
 
 // cluster_slots[c - 1] = clusters of c CTAs that can be resident at once (0 = size not allowed);
@@ -116,7 +118,7 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
             }
         }
         if ((int64_t)sizes.size() > item_cap) return;
-        const int64_t penalty = (merge_pass ? kMergePassPages : 0) + (C > 1 ? (kClusterPagesX5 * C + 4) / 5 : 0);
+        const int64_t penalty = (merge_pass ? kMergePassPages : 0) + (C > 1 ? ((rows <= 4 ? kPushClusterPagesX5 : kClusterPagesX5) * C + 4) / 5 : 0);
         if (std::max(longest, (total + slots - 1) / slots) + penalty >= best_cost) return;   // lower bound
         int64_t makespan = longest;
         if ((int64_t)sizes.size() > slots) {
