@@ -118,7 +118,8 @@ class ClockSampler:
 class Cycle:
     """Device-resident state of one configuration plus the graphs that replay a cycle."""
 
-    def __init__(self, name, seed, layers=None, device="cuda:0", decode_chunk=0, verify_chunk=0):
+    def __init__(self, name, seed, layers=None, device="cuda:0", decode_chunk=0, verify_chunk=0,
+                 kv_layout="hnd"):
         import torch
         from paper_2607_24260_b200 import kap, synth
         self.torch, self.kap, self.synth = torch, kap, synth
@@ -155,6 +156,13 @@ class Cycle:
         max_rows = int(w.n_q.max()) * (Hq // Hkv)
         self.ws_d = kap.Workspace(int(device.split(":")[1]), 8192, Hq // Hkv, B)
         self.ws_v = kap.Workspace(int(device.split(":")[1]), 8192, max_rows, B)
+        # token-major pools hold the same random values: the attention calls just read them through
+        # the other tensor map
+        self.pool_attn = self.pool
+        if kv_layout == "nhd":
+            self.pool_attn = self.pool.view(self.layers, w.num_pool_pages, 2, P, Hkv, d)
+            self.ws_d.set_kv_layout(kap.KV_NHD)
+            self.ws_v.set_kv_layout(kap.KV_NHD)
         self.info_d = self.ws_d.schedule(self.n_sel, None, Hq, Hkv, decode_chunk)
         self.info_v = self.ws_v.schedule(self.n_pages, w.n_q, Hq, Hkv, verify_chunk)
         self.chunks = (decode_chunk, verify_chunk)
@@ -171,14 +179,14 @@ class Cycle:
         kap = self.kap
         for step in range(self.k):
             for layer in range(self.layers):
-                kap.selected_decode_attn(self.q_dec[step, layer], self.pool[layer], self.d_plan_indptr,
+                kap.selected_decode_attn(self.q_dec[step, layer], self.pool_attn[layer], self.d_plan_indptr,
                                          self.d_plan_phys, self.d_plan_logical, self.d_ctx,
                                          self.out_dec[step, layer], self.ws_d)
 
     def enqueue_verify(self):
         kap = self.kap
         for layer in range(self.layers):
-            kap.verify_attn(self.q_ver[layer], self.d_q_indptr, self.pool[layer], self.d_bt_indptr,
+            kap.verify_attn(self.q_ver[layer], self.d_q_indptr, self.pool_attn[layer], self.d_bt_indptr,
                             self.d_bt_pages, self.d_ctx, self.out_ver[layer], self.ws_v)
 
     def capture(self):
@@ -225,7 +233,7 @@ class Cycle:
         for ws in (self.ws_d, self.ws_v):
             ws.close()
         self.graph_d = self.graph_v = None
-        self.pool = self.q_dec = self.q_ver = self.out_dec = self.out_ver = None
+        self.pool = self.pool_attn = self.q_dec = self.q_ver = self.out_dec = self.out_ver = None
         self.torch.cuda.empty_cache()
 
 
@@ -554,6 +562,8 @@ def main():
     ap.add_argument("--pdl", type=int, default=-1)
     ap.add_argument("--ctas-per-sm", type=int, default=-1)
     ap.add_argument("--early-kv", type=int, default=-1)
+    ap.add_argument("--kv-layout", default="hnd", choices=["hnd", "nhd"],
+                    help="pool layout given to the attention calls (default: head-major)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -572,7 +582,7 @@ def main():
     kap.set_launch_options(args.pdl, args.early_kv, args.ctas_per_sm, args.max_cluster, args.ring_slots)
     warmup = max(3, args.warmup)
 
-    cy = Cycle(args.config, seed=rank, layers=args.layers, device=dev, decode_chunk=args.decode_chunk,
+    cy = Cycle(args.config, seed=rank, layers=args.layers, device=dev, kv_layout=args.kv_layout, decode_chunk=args.decode_chunk,
                verify_chunk=args.verify_chunk)
     cy.capture()
     if dist:
@@ -600,7 +610,8 @@ def main():
         "data": "synthetic",
         "config": config_dict(w, k, cy.layers, {"parallelism": f"dp{world} (independent batches per GPU)",
                                                  "pdl": args.pdl, "max_cluster": args.max_cluster, "ring_slots": args.ring_slots,
-                                                 "ctas_per_sm": args.ctas_per_sm, "early_kv": args.early_kv}),
+                                                 "ctas_per_sm": args.ctas_per_sm, "early_kv": args.early_kv,
+                                                 "kv_layout": args.kv_layout}),
         "clocks": clocks.summary(),
         "e2e": {"value": world * w.batch * k / (e2e_ms * 1e-3), "unit": "tokens/s",
                 "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -54,6 +54,14 @@ typedef enum {
     KAP_ERR_DEVICE_INDEX = 6   /* a kernel met an out-of-range page or list index */
 } kap_status;
 
+/* Layout of one layer's paged KV pool.  HND (default): bf16 pool[page][2][Hkv][P][d], the K (or V)
+ * rows of one page and one KV head are contiguous.  NHD: bf16 pool[page][2][P][Hkv][d], token-major
+ * (what a fused QKV projection writes).  Same page size, same 65 536 bytes per page. */
+enum {
+    KAP_KV_HND = 0,
+    KAP_KV_NHD = 1
+};
+
 /* per-sequence plan flags (bit-or) written by kap_compile_plan */
 enum {
     KAP_PLAN_FULL = 1,         /* identity plan: the sequence takes full-context access */
@@ -174,6 +182,15 @@ kap_status kap_schedule_info(const kap_workspace* ws, int32_t* n_items, int32_t*
                              int32_t* cluster_size);
 
 /*
+ * kap_workspace_set_kv_layout - layout (KAP_KV_HND, the default, or KAP_KV_NHD) of the pools that
+ * later kap_selected_decode_attn / kap_verify_attn calls on this workspace will be given.  The
+ * paper does not fix a pool layout; both are read with the same tiles, bytes and arithmetic, and
+ * results are identical bit for bit.  Host only, no GPU work.  KAP_ERR_INVALID_ARG for a NULL
+ * workspace or an unknown layout.
+ */
+kap_status kap_workspace_set_kv_layout(kap_workspace* ws, int32_t kv_layout);
+
+/*
  * kap_selected_decode_attn - Section 3.2 "Selected-KV proposal".  For sequence b and query head h
  * (KV head g = h / G), with Vis(b) = the tokens t < ctx_len[b] of the plan's pages:
  *     z_t = sm_scale * <q[b,h,:], K[g,t,:]>,   out[b,h,:] = sum_t softmax_t(z) V[g,t,:],
@@ -259,6 +276,7 @@ kap_status kap_append_kv(
     int32_t* ctx_len,                  /* DEVICE [batch], read; updated when advance != 0 */
     int32_t advance,
     int32_t batch, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
+    int32_t kv_layout,                 /* KAP_KV_HND or KAP_KV_NHD: layout of kv_pool */
     int32_t* device_status,            /* DEVICE int32 or NULL */
     void* cuda_stream);
 

@@ -19,7 +19,7 @@ kap_append_kv_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ 
                      const int32_t* __restrict__ new_indptr, uint4* __restrict__ pool,
                      long long num_pool_pages, const int32_t* __restrict__ bt_indptr,
                      const int32_t* __restrict__ bt_pages, int32_t* ctx_len, int advance, int hkv,
-                     int32_t* status)
+                     int nhd, int32_t* status)
 {
     constexpr int kRowVec = kHeadDim * 2 / 16;                 // 16 uint4 per 128-element bf16 row
     const int b = blockIdx.x;
@@ -43,7 +43,10 @@ kap_append_kv_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ 
             continue;
         }
         const uint4* src = (kv ? v_new : k_new) + ((long long)(row0 + j) * hkv + g) * kRowVec + piece;
-        pool[page * page_vec + ((long long)(kv * hkv + g) * kPageSize + pos % kPageSize) * kRowVec + piece] = *src;
+        // row of (K|V, head g, slot) inside the page: head-major ("HND") or token-major ("NHD")
+        const long long row = nhd ? ((long long)kv * kPageSize + pos % kPageSize) * hkv + g
+                                  : (long long)(kv * hkv + g) * kPageSize + pos % kPageSize;
+        pool[page * page_vec + row * kRowVec + piece] = *src;
     }
     if (advance) {
         __syncthreads();                                         // every thread has read L
@@ -58,12 +61,14 @@ extern "C" kap_status kap_append_kv(
     const void* k_new, const void* v_new, const int32_t* new_indptr, void* kv_pool,
     int64_t num_pool_pages, const int32_t* bt_indptr, const int32_t* bt_pages, int32_t* ctx_len,
     int32_t advance, int32_t batch, int32_t num_kv_heads, int32_t head_dim, int32_t page_size,
-    int32_t* device_status, void* cuda_stream)
+    int32_t kv_layout, int32_t* device_status, void* cuda_stream)
 {
     using namespace kap;
     if (head_dim != kHeadDim || page_size != kPageSize)
         return fail(KAP_ERR_UNSUPPORTED, "head_dim %d / page_size %d (supported: 128 / 16)", head_dim, page_size);
     if (batch < 0 || num_kv_heads <= 0) return fail(KAP_ERR_INVALID_ARG, "batch %d / num_kv_heads %d", batch, num_kv_heads);
+    if (kv_layout != KAP_KV_HND && kv_layout != KAP_KV_NHD)
+        return fail(KAP_ERR_INVALID_ARG, "kv_layout %d (KAP_KV_HND = 0, KAP_KV_NHD = 1)", kv_layout);
     if (batch == 0) return KAP_OK;
     if (!k_new || !v_new || !kv_pool || !bt_indptr || !bt_pages || !ctx_len || num_pool_pages <= 0)
         return fail(KAP_ERR_INVALID_ARG, "NULL pointer or empty pool");
@@ -72,7 +77,7 @@ extern "C" kap_status kap_append_kv(
         return fail(KAP_ERR_INVALID_ARG, "k_new, v_new and kv_pool must be 16-byte aligned");
     kap_append_kv_kernel<<<(unsigned)batch, 256, 0, (cudaStream_t)cuda_stream>>>(
         (const uint4*)k_new, (const uint4*)v_new, new_indptr, (uint4*)kv_pool, num_pool_pages, bt_indptr,
-        bt_pages, ctx_len, advance, num_kv_heads, device_status);
+        bt_pages, ctx_len, advance, num_kv_heads, kv_layout == KAP_KV_NHD, device_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(KAP_ERR_CUDA, "kap_append_kv launch failed: %s", cudaGetErrorString(e));
     count_launch();

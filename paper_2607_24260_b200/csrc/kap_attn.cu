@@ -159,6 +159,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         " [%0], [%1, {%2, %3}], [%4], %5;"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int32_t x,
+                                            int32_t y, int32_t z, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
                                         uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -313,7 +320,11 @@ __device__ __forceinline__ void merge_group_cell(const AttnParams& p, const Merg
 // kPush selects the cluster reduction: false = every CTA reads its peers' shared memory between two
 // cluster barriers; true = every CTA pushes its cells into the owners' landing zones (few rows and
 // short lists only: the host picks it when every item of the launch qualifies).
-template <bool kPush>
+//
+// kNhd selects the pool layout: false = [page][2][Hkv][P][d] ("HND": a page-head's K rows are
+// contiguous; one 2-D tensor map over [rows][d]); true = [page][2][P][Hkv][d] ("NHD": token-major;
+// a 3-D tensor map (d, head, token row) whose 64 x 1 x 16 box lands in the same shared-memory tile).
+template <bool kPush, bool kNhd>
 __global__ void __launch_bounds__(kThreads, 3)
 kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
 {
@@ -418,13 +429,21 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         const int idx = k * n_groups + grp;                  // local id
         if (k < group_pages) {
             tail->slot_page[s] = idx;
-            const int y = id_phys[idx] * rows_per_page + item.kv_head * kPageSize;
             const uint32_t dst = smem_u32(ring + s * kPageHeadBytes);
             mbar_expect_tx(bar, kPageHeadBytes);
-            tma_load_2d(dst, &kv_map, 0, y, bar, policy);
-            tma_load_2d(dst + kHalfTileBytes, &kv_map, 64, y, bar, policy);
-            tma_load_2d(dst + kTileBytes, &kv_map, 0, y + v_row_off, bar, policy);
-            tma_load_2d(dst + kTileBytes + kHalfTileBytes, &kv_map, 64, y + v_row_off, bar, policy);
+            if (kNhd) {
+                const int z = id_phys[idx] * (2 * kPageSize);            // token row of the page's K
+                tma_load_3d(dst, &kv_map, 0, item.kv_head, z, bar, policy);
+                tma_load_3d(dst + kHalfTileBytes, &kv_map, 64, item.kv_head, z, bar, policy);
+                tma_load_3d(dst + kTileBytes, &kv_map, 0, item.kv_head, z + kPageSize, bar, policy);
+                tma_load_3d(dst + kTileBytes + kHalfTileBytes, &kv_map, 64, item.kv_head, z + kPageSize, bar, policy);
+            } else {
+                const int y = id_phys[idx] * rows_per_page + item.kv_head * kPageSize;
+                tma_load_2d(dst, &kv_map, 0, y, bar, policy);
+                tma_load_2d(dst + kHalfTileBytes, &kv_map, 64, y, bar, policy);
+                tma_load_2d(dst + kTileBytes, &kv_map, 0, y + v_row_off, bar, policy);
+                tma_load_2d(dst + kTileBytes + kHalfTileBytes, &kv_map, 64, y + v_row_off, bar, policy);
+            }
         } else {
             tail->slot_page[s] = -1;
             mbar_arrive(bar);                                // completes the phase with no bytes
@@ -803,9 +822,10 @@ EncodeTiledFn encode_tiled_fn() {
 // box = 16 rows x 64 columns (one half of a page-head's K or V), 128-byte swizzle.
 kap_status get_tensor_map(kap_workspace* ws, const void* pool, int64_t pages, int32_t hkv,
                           const CUtensorMap** out) {
+    const int32_t layout = ws->kv_layout;
     for (int i = 0; i < ws->map_count; ++i) {
         auto& s = ws->maps[i];
-        if (s.base == pool && s.pages == pages && s.hkv == hkv) {
+        if (s.base == pool && s.pages == pages && s.hkv == hkv && s.layout == layout) {
             *out = reinterpret_cast<const CUtensorMap*>(s.map);
             return KAP_OK;
         }
@@ -814,17 +834,31 @@ kap_status get_tensor_map(kap_workspace* ws, const void* pool, int64_t pages, in
     if (!enc) return fail(KAP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     const uint64_t rows = (uint64_t)pages * 2 * hkv * kPageSize;
     if (rows >= (1ull << 31)) return fail(KAP_ERR_UNSUPPORTED, "pool of %lld pages is too large", (long long)pages);
-    cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kPageSize};
-    cuuint32_t estr[2] = {1, 1};
     auto& slot = ws->maps[ws->map_next];
-    CUresult r = enc(reinterpret_cast<CUtensorMap*>(slot.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-                     const_cast<void*>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r;
+    if (layout == KAP_KV_NHD) {
+        // (d, head, token row): a head's row is 256 contiguous bytes, rows of one head are
+        // Hkv * 256 bytes apart; the box takes 64 columns of one head for the 16 tokens of a page
+        cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)hkv, (cuuint64_t)pages * 2 * kPageSize};
+        cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)hkv * kHeadDim * 2};
+        cuuint32_t box[3] = {64, 1, (cuuint32_t)kPageSize};
+        cuuint32_t estr[3] = {1, 1, 1};
+        r = enc(reinterpret_cast<CUtensorMap*>(slot.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                const_cast<void*>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+        cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
+        cuuint32_t box[2] = {64, (cuuint32_t)kPageSize};
+        cuuint32_t estr[2] = {1, 1};
+        r = enc(reinterpret_cast<CUtensorMap*>(slot.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                const_cast<void*>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
     if (r != CUDA_SUCCESS) return fail(KAP_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
-    slot.base = pool; slot.pages = pages; slot.hkv = hkv;
+    slot.base = pool; slot.pages = pages; slot.hkv = hkv; slot.layout = layout;
     *out = reinterpret_cast<const CUtensorMap*>(slot.map);
     ws->map_next = (ws->map_next + 1) % kap_workspace::kMapSlots;
     if (ws->map_count < kap_workspace::kMapSlots) ++ws->map_count;
@@ -844,15 +878,14 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     if (st != KAP_OK) return st;
     // function attributes are per device: set them once for the workspace's device
     if (!ws->attrs_set) {
-        cudaError_t ae = cudaFuncSetAttribute(kap_attn_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              smem_bytes_for(kMaxSlots));
-        if (ae == cudaSuccess)
-            ae = cudaFuncSetAttribute(kap_attn_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      smem_bytes_for(kMaxSlots));
-        if (ae != cudaSuccess) return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ae));
-        cudaFuncSetAttribute(kap_attn_split_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        cudaFuncSetAttribute(kap_attn_split_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        cudaGetLastError();
+        const void* variants[4] = {(const void*)kap_attn_split_kernel<false, false>, (const void*)kap_attn_split_kernel<true, false>,
+                                   (const void*)kap_attn_split_kernel<false, true>, (const void*)kap_attn_split_kernel<true, true>};
+        for (const void* fn : variants) {
+            cudaError_t ae = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(kMaxSlots));
+            if (ae != cudaSuccess) return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ae));
+            cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            cudaGetLastError();
+        }
         ws->attrs_set = 1;
     }
 
@@ -891,8 +924,11 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     cfg.numAttrs = n_attr;
     // few rows and short lists in every item (the proposal path): push-style cluster reduction
     const bool push = ws->cluster_size > 1 && ws->max_nq * p.G <= kPushRows && ws->max_chunk <= kPushIds;
-    if (push) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<true>, *map, p));
-    else KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<false>, *map, p));
+    const bool nhd = ws->kv_layout == KAP_KV_NHD;
+    if (push && nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<true, true>, *map, p));
+    else if (push) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<true, false>, *map, p));
+    else if (nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<false, true>, *map, p));
+    else KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<false, false>, *map, p));
     g_launches.fetch_add(1);
     if (ws->n_merge_groups > 0) {
         const int rows = ws->max_nq * p.G;
@@ -1007,10 +1043,10 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     KAP_CUDA(cudaSetDevice(ws->device));
     const int ring_slots = g_ring_slots.load();
     const int smem = smem_bytes_for(ring_slots);
-    cudaFuncSetAttribute(kap_attn_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(kap_attn_split_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          smem_bytes_for(kMaxSlots));
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel<false>, kThreads, smem) != cudaSuccess || occ < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel<false, false>, kThreads, smem) != cudaSuccess || occ < 1)
         occ = 1;
     const int want = g_ctas_per_sm.load();
     const int per_sm = want > 0 ? std::min(want, occ) : occ;
@@ -1018,7 +1054,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     ws->ring_slots = ring_slots;
     ws->ctas_per_wave = per_sm * ws->sm_count;
     int32_t slots[kMaxCluster] = {ws->ctas_per_wave};
-    cudaFuncSetAttribute(kap_attn_split_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    cudaFuncSetAttribute(kap_attn_split_kernel<false, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     cudaGetLastError();
     for (int c = 2; c <= kMaxCluster; ++c) {
         if (c > g_max_cluster.load()) continue;
@@ -1031,7 +1067,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         cc.dynamicSmemBytes = smem;
         cc.attrs = ca; cc.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel<false>, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
+        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel<false, false>, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
         slots[c - 1] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
     }
     // a one-wave schedule leaves a third of the SM's CTA slots to the next kernel's early CTAs
@@ -1167,6 +1203,14 @@ extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, 
     return KAP_OK;
 }
 
+extern "C" kap_status kap_workspace_set_kv_layout(kap_workspace* ws, int32_t kv_layout) {
+    if (!ws) return fail(KAP_ERR_INVALID_ARG, "NULL workspace");
+    if (kv_layout != KAP_KV_HND && kv_layout != KAP_KV_NHD)
+        return fail(KAP_ERR_INVALID_ARG, "kv_layout %d (KAP_KV_HND = 0, KAP_KV_NHD = 1)", kv_layout);
+    ws->kv_layout = kv_layout;
+    return KAP_OK;
+}
+
 extern "C" int64_t kap_launch_count(void) { return g_launches.load(); }
 
 #ifdef KAP_TRACE
@@ -1280,7 +1324,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
         if (!g_static_ready[dev]) {
             void* ptr = nullptr;
             KAP_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
-            KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel<false>,
+            KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel<false, false>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           smem_bytes_for(kMaxSlots)));
             g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
@@ -1335,7 +1379,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
     g_launches.fetch_add(1);
     // plain launches: the work list was written by the kernel just before, so the split kernel
     // must not start early
-    kap_attn_split_kernel<false><<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
+    kap_attn_split_kernel<false, false><<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
     KAP_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     if (num_splits > 1) {

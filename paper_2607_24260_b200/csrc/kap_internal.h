@@ -51,6 +51,7 @@ struct kap_workspace {
     int32_t batch = 0, n_items = 0, n_groups = 0, n_merge_groups = 0, max_chunk = 0;
     int32_t ctas_per_wave = 0, row_tiles = 1, num_q_heads = 0, num_kv_heads = 0;
     int32_t has_nq = 0;            // schedule was made with an n_q array (verification path)
+    int32_t kv_layout = 0;         // KAP_KV_HND / KAP_KV_NHD: layout of the pools given to the attention calls
     int32_t plain_next = 0;        // the page lists were just rewritten on the device: launch the
                                    // next attention kernel as an ordinary (fully ordered) one
     int64_t total_rows = 0;        // sum over sequences of n_q
@@ -69,7 +70,7 @@ struct kap_workspace {
     int32_t* h_status = nullptr;             // pinned read-back
     void* upload_event = nullptr;            // cudaEvent_t: last schedule upload done
     // cached tensor maps, keyed by (pool pointer, pages, Hkv)
-    struct MapSlot { const void* base; int64_t pages; int32_t hkv; alignas(64) unsigned char map[128]; };
+    struct MapSlot { const void* base; int64_t pages; int32_t hkv, layout; alignas(64) unsigned char map[128]; };
     static constexpr int kMapSlots = 64;
     MapSlot* maps = nullptr;
     int32_t map_next = 0, map_count = 0;

@@ -16,6 +16,7 @@ from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_DEVICE_INDEX = range(7)
 PLAN_FULL, PLAN_OVER_BUDGET, PLAN_S_HIGH, PLAN_MOVES_WITH_LENGTH = 1, 2, 4, 8
+KV_HND, KV_NHD = 0, 1
 
 _i32p, _f32p, _u8p, _vp = C.POINTER(C.c_int32), C.POINTER(C.c_float), C.POINTER(C.c_uint8), C.c_void_p
 
@@ -46,7 +47,8 @@ SIGNATURES = {
                                                   C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                   C.c_float, C.c_int32, _vp, _vp, _vp, _vp]),
     "kap_append_kv": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int64, _vp, _vp, _vp, C.c_int32, C.c_int32,
-                                C.c_int32, C.c_int32, C.c_int32, _vp, _vp]),
+                                C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp]),
+    "kap_workspace_set_kv_layout": (C.c_int, [_vp, C.c_int32]),
     "kap_top3_accept": (C.c_int, [_vp, C.c_int64, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
                                   _vp, _vp]),
     "kap_phase_model": (C.c_int, [C.c_double] * 6 + [C.POINTER(C.c_double)]),
@@ -233,6 +235,12 @@ def _dptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
 
 
+def _pool_shape(kv_pool, ws):
+    """(pages, Hkv, P) of a pool tensor in the layout the workspace is set to"""
+    pages, _, a, b, _ = kv_pool.shape
+    return (pages, b, a) if getattr(ws, "kv_layout", KV_HND) == KV_NHD else (pages, a, b)
+
+
 class Workspace:
     """kap_workspace: split-K schedule + partial-result buffers for one launch shape."""
 
@@ -258,6 +266,11 @@ class Workspace:
                                   _stream_ptr(stream)))
         return self.info()
 
+    def set_kv_layout(self, kv_layout):
+        """KV_HND (default): pools are [pages, 2, Hkv, P, d]; KV_NHD: [pages, 2, P, Hkv, d]."""
+        _check(lib().kap_workspace_set_kv_layout(self._h, int(kv_layout)))
+        self.kv_layout = int(kv_layout)
+
     def info(self):
         v = [C.c_int32(0) for _ in range(5)]
         _check(lib().kap_schedule_info(self._h, *[C.byref(x) for x in v]))
@@ -274,7 +287,7 @@ def selected_decode_attn(q, kv_pool, plan_indptr, plan_phys_pages, plan_logical_
     [pages, 2, Hkv, P, d]; plan arrays and ctx_len int32 device tensors; plan_token_masks an
     optional uint16 device tensor (one word per listed page) for token-granular visibility."""
     B, Hq, d = q.shape
-    pages, _, Hkv, P, _ = kv_pool.shape
+    pages, Hkv, P = _pool_shape(kv_pool, ws)
     sm_scale = float(d) ** -0.5 if sm_scale is None else float(sm_scale)
     _check(lib().kap_selected_decode_attn(
         _dptr(q), _dptr(kv_pool), int(pages), _dptr(plan_indptr), _dptr(plan_phys_pages),
@@ -287,7 +300,7 @@ def verify_attn(q, q_indptr, kv_pool, bt_indptr, bt_pages, ctx_len, out, ws: Wor
                 sm_scale=None, stream=None):
     """kap_verify_attn on torch CUDA tensors: q/out bf16 [sum n_q, Hq, d]."""
     _, Hq, d = q.shape
-    pages, _, Hkv, P, _ = kv_pool.shape
+    pages, Hkv, P = _pool_shape(kv_pool, ws)
     sm_scale = float(d) ** -0.5 if sm_scale is None else float(sm_scale)
     _check(lib().kap_verify_attn(
         _dptr(q), _dptr(q_indptr), _dptr(kv_pool), int(pages), _dptr(bt_indptr), _dptr(bt_pages),
@@ -313,13 +326,17 @@ def selected_decode_attn_static(q, kv_pool, plan_indptr, plan_phys_pages, plan_l
 
 
 def append_kv(k_new, v_new, kv_pool, bt_indptr, bt_pages, ctx_len, new_indptr=None, advance=True,
-              device_status=None, stream=None):
+              device_status=None, stream=None, kv_layout=KV_HND):
     """kap_append_kv: write the new tokens' K/V rows (bf16 [sum n_new, Hkv, d]) into the paged pool
-    at positions ctx_len[b] .. and, with advance, bump ctx_len on the device."""
-    pages, _, Hkv, P, d = kv_pool.shape
+    at positions ctx_len[b] .. and, with advance, bump ctx_len on the device.  kv_pool has shape
+    [pages, 2, Hkv, P, d] (KV_HND) or [pages, 2, P, Hkv, d] (KV_NHD)."""
+    if kv_layout == KV_NHD:
+        pages, _, P, Hkv, d = kv_pool.shape
+    else:
+        pages, _, Hkv, P, d = kv_pool.shape
     _check(lib().kap_append_kv(_dptr(k_new), _dptr(v_new), _dptr(new_indptr), _dptr(kv_pool), int(pages),
                                _dptr(bt_indptr), _dptr(bt_pages), _dptr(ctx_len), int(bool(advance)),
-                               int(ctx_len.shape[0]), Hkv, d, P, _dptr(device_status),
+                               int(ctx_len.shape[0]), Hkv, d, P, int(kv_layout), _dptr(device_status),
                                _stream_ptr(stream)))
 
 

@@ -33,8 +33,13 @@ def u16(a) -> torch.Tensor:
     return torch.from_numpy(np.array(a, dtype=np.uint16, copy=True).view(np.int16)).to(DEV)
 
 
+def to_nhd(pool_bits: np.ndarray) -> np.ndarray:
+    """[pages, 2, Hkv, P, d] (head-major) -> [pages, 2, P, Hkv, d] (token-major), same values"""
+    return np.ascontiguousarray(pool_bits.transpose(0, 1, 3, 2, 4))
+
+
 def run_decode(q_bits, pool_dev, plan, ctx_len, Hq=32, Hkv=8, max_chunk_pages=0, ws=None,
-               logical=True, sm_scale=None, masks=None):
+               logical=True, sm_scale=None, masks=None, kv_layout=kap.KV_HND):
     """Library proposal-path attention.  q_bits [B, Hq, d] uint16; pool_dev torch bf16
     [pages, 2, Hkv, P, d]; plan = dict from a plan compiler; masks = optional uint16 word per
     listed page (token-granular visibility).  Returns (out f64, lse f64)."""
@@ -43,6 +48,7 @@ def run_decode(q_bits, pool_dev, plan, ctx_len, Hq=32, Hkv=8, max_chunk_pages=0,
     own = ws is None
     if own:
         ws = kap.Workspace(max_rows_per_item=Hq // Hkv, max_batch=max(B, 1))
+        ws.set_kv_layout(kv_layout)
     ws.schedule(n, None, Hq, Hkv, max_chunk_pages)
     q = bits_to_dev(q_bits)
     out = torch.full_like(q, float("nan"))
@@ -59,7 +65,7 @@ def run_decode(q_bits, pool_dev, plan, ctx_len, Hq=32, Hkv=8, max_chunk_pages=0,
 
 
 def run_verify(q_bits, n_q, pool_dev, bt_indptr, bt_pages, ctx_len, Hq=32, Hkv=8,
-               max_chunk_pages=0, ws=None, page=16, sm_scale=None):
+               max_chunk_pages=0, ws=None, page=16, sm_scale=None, kv_layout=kap.KV_HND):
     """Library verification attention.  q_bits [sum n_q, Hq, d] uint16."""
     n_q = np.asarray(n_q, dtype=np.int32)
     B = n_q.shape[0]
@@ -68,6 +74,7 @@ def run_verify(q_bits, n_q, pool_dev, bt_indptr, bt_pages, ctx_len, Hq=32, Hkv=8
     own = ws is None
     if own:
         ws = kap.Workspace(max_rows_per_item=int(n_q.max()) * (Hq // Hkv), max_batch=max(B, 1))
+        ws.set_kv_layout(kv_layout)
     n_pages = (np.asarray(ctx_len, dtype=np.int64) + page - 1) // page
     ws.schedule(n_pages, n_q, Hq, Hkv, max_chunk_pages)
     q = bits_to_dev(q_bits)
