@@ -421,7 +421,36 @@ def time_extras(cy: Cycle, vocab: int = 128256, iters: int = 20):
     out["growing_plan_decode_us_per_layer"] = timed(masked)
     ws.check()
     ws.close()
+    # full-context decode (the fallback path: identity plan, one query row over the whole block
+    # table), the t_full of the paper's cost model
+    ws = kap.Workspace(int(dev.split(":")[1]), 8192, w.num_q_heads // w.num_kv_heads, w.batch)
+    ws.schedule(cy.n_pages, None, w.num_q_heads, w.num_kv_heads)
+
+    def full():
+        layer = turn[0] % cy.layers
+        kap.selected_decode_attn(cy.q_dec[0, layer], cy.pool[layer], cy.d_bt_indptr, cy.d_bt_pages, None,
+                                 cy.d_ctx, o, ws)
+        turn[0] += 1
+    out["full_decode_us_per_layer"] = timed(full)
+    ws.check()
+    ws.close()
     return out
+
+
+def phase_report(kap, k, t_sel, t_verify, t_full):
+    """The paper's phase boundary (Eqs. 6-13) on this run's measured per-layer attention times,
+    with the weight terms at zero (attention only): s_time = t_sel / t_full plays the part of the
+    retained ratio, the plan pays off iff the acceptance rate h exceeds the break-even value."""
+    s_time = t_sel / t_full
+    rep = {"k": k, "t_sel_us": t_sel, "t_verify_us": t_verify, "t_full_us": t_full,
+           "s_time": s_time,
+           # (1 + k h) t_full = k t_sel + t_verify  (Eq. 6 = Eq. 7 with the measured verifier time)
+           "break_even_h": max(0.0, (k * t_sel + t_verify - t_full) / (k * t_full))}
+    for h in (0.6, 0.8, 1.0):
+        m = kap.phase_model(k, h, min(s_time, 1.0), 0.0, 0.0, t_full)
+        rep[f"model_speedup_h{h}"] = m["speedup"]                       # verifier at t_full (Eq. 7)
+        rep[f"measured_speedup_h{h}"] = (1 + k * h) * t_full / (k * t_sel + t_verify)
+    return rep
 
 
 # ---------------------------------------------------------------------------------- CPU baseline
@@ -626,6 +655,8 @@ def main():
     }
     if extras:
         line["other_calls"] = extras
+        line["phase"] = phase_report(kap, cy.k, res["us_per_layer_decode"], res["us_per_layer_verify"],
+                                     extras["full_decode_us_per_layer"])
     cy.free()
 
     if rank == 0 and world == 1 and not args.no_sweep and args.config == "c2":
