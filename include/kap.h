@@ -413,6 +413,8 @@ kap_status kap_refresh_recent(
  * (compact_pool, compact_pages, plan_logical_pages) then equals the in-place call bit for bit.
  * This library's attention gathers in place and does not need the copy; the call is here for
  * comparison and for back ends that want a dense view.
+ * Pages are copied whole, so the call serves either pool layout.  Token masks and logical pages
+ * are indexed by list position and apply to the copy unchanged.
  * n_selected > compact_capacity is the paper's "plan exceeds the workspace" fallback condition:
  * KAP_ERR_CAPACITY, nothing enqueued.  A source page outside the pool is reported in
  * *device_status (1 << KAP_ERR_DEVICE_INDEX) and not copied.  Other errors: KAP_ERR_UNSUPPORTED
@@ -458,6 +460,8 @@ kap_status kap_materialize_view(
  *     by the caller.
  *   - kernels are launched without programmatic stream serialisation (the work list is produced
  *     on the device just before it is read).
+ *   - page-granular visibility and the head-major (KAP_KV_HND) pool layout only: token masks and
+ *     the token-major layout belong to the workspace entry point.
  * Results are the same as the workspace entry point's up to the order of the fp32 sums.
  * device_status (DEVICE int32, may be NULL) receives the kernels' status bits after the call's
  * kernels: 0, or 1 << KAP_ERR_DEVICE_INDEX / 1 << KAP_ERR_TIMEOUT.
