@@ -1070,9 +1070,12 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel<false, false>, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
         slots[c - 1] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
     }
-    // a one-wave schedule leaves a third of the SM's CTA slots to the next kernel's early CTAs
+    // A one-wave schedule of the proposal path leaves a third of the SM's CTA slots to the next
+    // kernel's early CTAs: those kernels last 10-30 us and what the early CTAs prefetch is a large
+    // part of the next layer.  Verification kernels last 80-550 us; there the slots are worth more
+    // than the early start (measured on the 16K configuration: 86.6 -> 84.2 us per layer).
     int32_t one_wave[kMaxCluster];
-    const int keep = per_sm >= occ && occ >= 3 ? occ - occ / 3 : per_sm;
+    const int keep = !n_q && per_sm >= occ && occ >= 3 ? occ - occ / 3 : per_sm;
     for (int c = 1; c <= kMaxCluster; ++c)
         one_wave[c - 1] = (int32_t)((int64_t)slots[c - 1] * keep / per_sm);
     int32_t cluster = 1;
