@@ -2,16 +2,18 @@
 // "Selected-KV proposal") and kap_verify_attn (Section 3.2, "Full-context verification") of the
 // KAP paper, plus the log-sum-exp merge of the splits.
 //
-// One CTA = one work item = a contiguous slice of one sequence's page list for one KV head.
+// One work item = a contiguous slice of one sequence's page list for one KV head, run by a
+// thread-block cluster of C CTAs (C = 1: a single CTA), each of which takes an even part of it.
 //   * each page's K and V rows for this KV head arrive by TMA tensor loads (cp.async.bulk.tensor,
 //     128-byte swizzle) in a ring of shared-memory page slots, completion tracked by mbarriers;
-//     one elected lane per warp group keeps the group's slots refilled;
-//   * four warps each own one 16-row tile of query rows (rows = n_q * G: the G query heads of
+//     the last warp of a warp group to finish a page refills its slot;
+//   * the warps share the item's query rows in 16-row tiles (rows = n_q * G: the G query heads of
 //     the KV head's group times the n_q query tokens, so every K/V byte is read from HBM once and
 //     shared by all of them), compute S = Q K^T and O += P V with bf16 mma.sync tiles and fp32
 //     accumulators, and keep a base-2 online softmax per row in registers;
-//   * the warps' states are combined through shared memory and the CTA writes either the final
-//     bf16 output (single split) or an un-normalised fp32 partial (m, l, O) for the merge pass.
+//   * the warps' states are combined through shared memory, the cluster's CTAs reduce theirs
+//     through distributed shared memory, and the result is either the final bf16 output (the
+//     item is the whole list) or an un-normalised fp32 partial (m, l, O) for the merge pass.
 // The proposal path is the n_q = 1 case of the same kernel; the causal rule "row j sees tokens
 // t <= L - n_q + j" covers both paths.
 //
@@ -314,8 +316,8 @@ __device__ __forceinline__ void merge_group_cell(const AttnParams& p, const Merg
 // Shared-memory ring: 8 page slots of 8 KiB (K tile then V tile, each two 64-column halves in the
 // TMA 128-byte swizzle).  With RT row tiles the 4 warps form 4/RT warp groups; page i of the slice
 // belongs to group i mod (4/RT) and is consumed by that group's RT warps (one per row tile).  Each
-// group owns 8/(4/RT) slots as a private ring; lane 0 of the group's first warp refills a slot as
-// soon as all RT warps have released it, so every group always has its whole ring in flight.
+// group owns 8/(4/RT) slots as a private ring; the last of its RT warps to release a slot refills
+// it at once, so every group always has its whole ring in flight and no warp waits for a partner.
 //
 // kPush selects the cluster reduction: false = every CTA reads its peers' shared memory between two
 // cluster barriers; true = every CTA pushes its cells into the owners' landing zones (few rows and
