@@ -56,7 +56,12 @@ def _run_library(w, pool, q, plan):
     kap.verify_attn(z_v, d["q_indptr"], pool, d["bt_indptr"], d["bt_pages"], d["ctx"], torch.zeros_like(q), ws_v, lse=zl_v)
     ws_d.check()
     ws_v.check()
-    res = dict(qd=qd, out_d=out_d, out_v=out_v, lse_d=lse_d.double().cpu().numpy(),
+    # the same property under the plan's token masks: only the selected union is visible
+    zl_m = torch.zeros_like(lse_d)
+    kap.selected_decode_attn(z_d, pool, d["indptr"], d["phys"], d["logical"], d["ctx"], torch.zeros_like(qd), ws_d,
+                             lse=zl_m, plan_token_masks=gu.u16(plan["plan_token_masks"]))
+    ws_d.check()
+    res = dict(zl_m=zl_m.double().cpu().numpy(), qd=qd, out_d=out_d, out_v=out_v, lse_d=lse_d.double().cpu().numpy(),
                lse_v=lse_v.double().cpu().numpy(), zl_d=zl_d.double().cpu().numpy(),
                zl_v=zl_v.double().cpu().numpy(), info_d=info_d, info_v=info_v)
     ws_d.close()
@@ -75,7 +80,8 @@ def test_full_size_configuration(name):
     w, pool, q = _device_case(name)
     plan = kap.compile_workload(w)
     ref_plan = orc.compile_workload(w)
-    for k in ("plan_indptr", "plan_logical_pages", "plan_phys_pages", "plan_flags", "selected_tokens"):
+    for k in ("plan_indptr", "plan_logical_pages", "plan_phys_pages", "plan_flags", "selected_tokens",
+              "plan_token_masks"):
         np.testing.assert_array_equal(plan[k], ref_plan[k])
     r = _run_library(w, pool, q, plan)
     G = w.num_q_heads // w.num_kv_heads
@@ -89,6 +95,9 @@ def test_full_size_configuration(name):
         lp = plan["plan_logical_pages"][plan["plan_indptr"][b]:plan["plan_indptr"][b + 1]]
         vis = int(np.minimum(16, L - lp.astype(np.int64) * 16).sum())
         np.testing.assert_allclose(r["zl_d"][b], np.log(vis), atol=3e-5, err_msg=f"{name} decode seq {b}")
+        # token-granular: exactly the tokens of the selected union (the oracle's count)
+        np.testing.assert_allclose(r["zl_m"][b], np.log(int(ref_plan["selected_tokens"][b])), atol=3e-5,
+                                   err_msg=f"{name} masked decode seq {b}")
         for j in range(int(w.n_q[b])):
             row = int(w.q_indptr[b]) + j
             np.testing.assert_allclose(r["zl_v"][row], np.log(L - int(w.n_q[b]) + j + 1), atol=3e-5,
