@@ -74,8 +74,10 @@ def test_growth_loop_in_one_graph(seed, steps):
     moves = (g["plan_flags"] & kap.PLAN_MOVES_WITH_LENGTH) != 0
     assert moves.any() and not moves.all()
     rng = synth.rng_for(seed, "growth-loop")
-    q_bits, pool_bits = synth.host_qkv(w, seed, q_rows=(steps + 1) * B, q_std=4.0)
-    q_bits = q_bits.reshape(steps + 1, B, Hq, d)
+    # two attention calls per step (two "layers" on the same pool): the first launch after a
+    # refresh is an ordinary one, the second overlaps it through programmatic dependent launch
+    q_bits, pool_bits = synth.host_qkv(w, seed, q_rows=(steps + 1) * 2 * B, q_std=4.0)
+    q_bits = q_bits.reshape(steps + 1, 2, B, Hq, d)
     k_new = synth.normal_bf16((steps, B, Hkv, d), 0.5, rng)
     v_new = synth.normal_bf16((steps, B, Hkv, d), 0.5, rng)
     dev = _Device(w, g, pool_bits)
@@ -85,12 +87,14 @@ def test_growth_loop_in_one_graph(seed, steps):
 
     def run():
         dev.refresh()                                       # step 0: the length the plan was compiled at
-        dev.decode(d_q[0], d_out[0])
+        dev.decode(d_q[0, 0], d_out[0, 0])
+        dev.decode(d_q[0, 1], d_out[0, 1])
         for t in range(steps):
             kap.append_kv(d_k[t], d_v[t], dev.pool, dev.bt_indptr, dev.bt_pages, dev.ctx, advance=True,
                           device_status=status)
             dev.refresh()
-            dev.decode(d_q[t + 1], d_out[t + 1])
+            dev.decode(d_q[t + 1, 0], d_out[t + 1, 0])
+            dev.decode(d_q[t + 1, 1], d_out[t + 1, 1])
 
     stream = torch.cuda.Stream()
     stream.wait_stream(torch.cuda.current_stream())
@@ -127,10 +131,11 @@ def test_growth_loop_in_one_graph(seed, steps):
                 assert S == _fresh(w, b, int(L[b]))[0], (t, b)      # == Algorithm 1 at this length
             sets.append(S)
         indptr, phys, logical, masks = _lists_from_tokens(sets, w)
-        ref, _, _, _ = orc.selected_decode_attn(q_bits[t], host_pool, indptr, phys, logical, L,
-                                                plan_token_masks=masks)
-        assert_close(got[t], ref, what=f"step {t}")
-        assert gu.normalised_error(got[t], ref) <= 2e-2
+        for layer in range(2):
+            ref, _, _, _ = orc.selected_decode_attn(q_bits[t, layer], host_pool, indptr, phys, logical, L,
+                                                    plan_token_masks=masks)
+            assert_close(got[t, layer], ref, what=f"step {t} call {layer}")
+            assert gu.normalised_error(got[t, layer], ref) <= 2e-2
     # after the last step the device arrays list exactly that token set, no token twice
     for b in range(B):
         listed = dev.listed_tokens(b)
