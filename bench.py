@@ -272,7 +272,10 @@ def summarise(cy: Cycle, steps, total_ms, dec_ms, ver_ms, n_ranks=1):
 def time_e2e(cy: Cycle, steps, warmup):
     """The same cycle through the C ABI from HOST buffers: compile + schedule on the host, pinned
     host -> device copies of the plan arrays, context lengths and every query, the two graph
-    segments, device -> host copies of every attention output; synchronised per step."""
+    segments, device -> host copies of every attention output; synchronised per step.  Inside a
+    step a second stream carries the copies that the running segment does not need: the
+    verification queries go up while the proposal passes run, the proposal outputs come down while
+    the verification pass runs."""
     torch, kap, w = cy.torch, cy.kap, cy.w
     pin = lambda t: torch.empty(t.shape, dtype=t.dtype).pin_memory()
     h_q_dec, h_q_ver = pin(cy.q_dec), pin(cy.q_ver)
@@ -288,6 +291,9 @@ def time_e2e(cy: Cycle, steps, warmup):
     h2d = (h_q_dec.numel() + h_q_ver.numel()) * 2 + (h_indptr.numel() + 2 * n_plan + h_ctx.numel()) * 4
     d2h = (h_out_dec.numel() + h_out_ver.numel()) * 2
 
+    side = torch.cuda.Stream(device=cy.dev)
+    up_done, qver_done, dec_done = (torch.cuda.Event() for _ in range(3))
+
     def one_step():
         plan = kap.compile_workload(w)                      # host: Algorithm 1
         n = int(plan["plan_indptr"][-1])
@@ -301,10 +307,19 @@ def time_e2e(cy: Cycle, steps, warmup):
         cy.d_plan_logical[:n].copy_(h_logical[:n], non_blocking=True)
         cy.d_ctx.copy_(h_ctx, non_blocking=True)
         cy.q_dec.copy_(h_q_dec, non_blocking=True)
-        cy.q_ver.copy_(h_q_ver, non_blocking=True)
+        main = torch.cuda.current_stream()
+        up_done.record(main)
+        with torch.cuda.stream(side):
+            side.wait_event(up_done)                        # after the proposal queries: same PCIe direction
+            cy.q_ver.copy_(h_q_ver, non_blocking=True)
+            qver_done.record(side)
         cy.graph_d.replay()
+        dec_done.record(main)
+        with torch.cuda.stream(side):
+            side.wait_event(dec_done)
+            h_out_dec.copy_(cy.out_dec, non_blocking=True)
+        main.wait_event(qver_done)
         cy.graph_v.replay()
-        h_out_dec.copy_(cy.out_dec, non_blocking=True)
         h_out_ver.copy_(cy.out_ver, non_blocking=True)
         torch.cuda.synchronize()
 
