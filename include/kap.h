@@ -296,6 +296,10 @@ kap_status kap_append_kv(
  *   next_token[b]  top3[row m][0]: the verifier's own best token at the first position that was not
  *                  accepted, or at the bonus position when all k_b were (the paper leaves the
  *                  choice of the carry open; this is the reading used here).
+ *   ctx_len[b]     (optional commit step) reduced by k_b - m: with the proposals' K/V appended
+ *                  during the cycle, ctx_len counts all k_b of them on entry and only the accepted
+ *                  ones on return; the rejected tokens' slots are overwritten by the next
+ *                  cycle's appends.  The carry token is not in the cache yet.
  * logits: DEVICE fp32, row r starts at logits + r * row_stride.  All outputs DEVICE int32; top3 is
  * [total_rows, 3] and is required (it is also the scratch between the two kernels).
  * Errors: KAP_ERR_INVALID_ARG (NULL pointer, vocab < 3, row_stride < vocab, negative counts),
@@ -309,6 +313,7 @@ kap_status kap_top3_accept(
     int32_t* top3,                     /* DEVICE out [total_rows, 3] */
     int32_t* accepted,                 /* DEVICE out [batch] */
     int32_t* next_token,               /* DEVICE out [batch] */
+    int32_t* ctx_len,                  /* DEVICE in/out [batch], or NULL: no commit */
     void* cuda_stream);
 
 /*

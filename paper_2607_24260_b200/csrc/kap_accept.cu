@@ -124,7 +124,8 @@ kap_top3_rows_kernel(const float* __restrict__ logits, long long row_stride, int
 
 __global__ void kap_accept_prefix_kernel(const int32_t* __restrict__ top3, const int32_t* __restrict__ row_indptr,
                                          const int32_t* __restrict__ proposed, int batch,
-                                         int32_t* __restrict__ accepted, int32_t* __restrict__ next_token)
+                                         int32_t* __restrict__ accepted, int32_t* __restrict__ next_token,
+                                         int32_t* ctx_len)
 {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
@@ -139,6 +140,9 @@ __global__ void kap_accept_prefix_kernel(const int32_t* __restrict__ top3, const
     }
     accepted[b] = m;
     next_token[b] = top3[(long long)(r0 + m) * 3];
+    // commit: the K/V of the n - 1 - m rejected proposals falls off the end of the context (their
+    // slots are overwritten by the next cycle's appends)
+    if (ctx_len) ctx_len[b] -= n - 1 - m;
 }
 
 }  // namespace
@@ -147,7 +151,7 @@ __global__ void kap_accept_prefix_kernel(const int32_t* __restrict__ top3, const
 extern "C" kap_status kap_top3_accept(
     const float* logits, int64_t row_stride, const int32_t* row_indptr, const int32_t* proposed,
     int32_t batch, int32_t total_rows, int32_t vocab, int32_t* top3, int32_t* accepted,
-    int32_t* next_token, void* cuda_stream)
+    int32_t* next_token, int32_t* ctx_len, void* cuda_stream)
 {
     using namespace kap;
     if (batch < 0 || total_rows < 0 || vocab < 3 || row_stride < vocab)
@@ -180,7 +184,7 @@ extern "C" kap_status kap_top3_accept(
     if (e == cudaSuccess) {
         count_launch();
         kap_accept_prefix_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, stream>>>(top3, row_indptr, proposed,
-                                                                                    batch, accepted, next_token);
+                                                                                    batch, accepted, next_token, ctx_len);
         e = cudaGetLastError();
         if (e == cudaSuccess) count_launch();
     }

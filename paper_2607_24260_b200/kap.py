@@ -50,7 +50,7 @@ SIGNATURES = {
                                 C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp]),
     "kap_workspace_set_kv_layout": (C.c_int, [_vp, C.c_int32]),
     "kap_top3_accept": (C.c_int, [_vp, C.c_int64, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
-                                  _vp, _vp]),
+                                  _vp, _vp, _vp]),
     "kap_phase_model": (C.c_int, [C.c_double] * 6 + [C.POINTER(C.c_double)]),
     "kap_materialize_view": (C.c_int, [_vp, C.c_int64, _vp, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                        _vp, C.c_int64, _vp, _vp, _vp]),
@@ -340,14 +340,14 @@ def append_kv(k_new, v_new, kv_pool, bt_indptr, bt_pages, ctx_len, new_indptr=No
                                _stream_ptr(stream)))
 
 
-def top3_accept(logits, row_indptr, proposed, top3, accepted, next_token, stream=None):
+def top3_accept(logits, row_indptr, proposed, top3, accepted, next_token, stream=None, ctx_len=None):
     """kap_top3_accept on torch CUDA tensors: logits fp32 [rows, vocab] (row stride taken from the
     tensor), int32 row_indptr [B+1], proposed [rows]; outputs int32 top3 [rows, 3], accepted [B],
-    next_token [B]."""
+    next_token [B].  ctx_len (int32 [B], optional) is reduced by the number of rejected proposals."""
     rows, vocab = logits.shape
     _check(lib().kap_top3_accept(_dptr(logits), int(logits.stride(0)), _dptr(row_indptr), _dptr(proposed),
                                  int(row_indptr.shape[0]) - 1, int(rows), int(vocab), _dptr(top3),
-                                 _dptr(accepted), _dptr(next_token), _stream_ptr(stream)))
+                                 _dptr(accepted), _dptr(next_token), _dptr(ctx_len), _stream_ptr(stream)))
 
 
 PHASE_FIELDS = ("cost_full", "cost_base", "cost_plan", "speedup", "slack", "kv_crit", "beneficial",

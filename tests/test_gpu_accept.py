@@ -18,8 +18,12 @@ def _run(logits_np, indptr, proposed, stride_pad=0):
     top3 = torch.full((rows, 3), -7, dtype=torch.int32, device=gu.DEV)
     acc = torch.full((len(indptr) - 1,), -7, dtype=torch.int32, device=gu.DEV)
     nxt = torch.full((len(indptr) - 1,), -7, dtype=torch.int32, device=gu.DEV)
-    kap.top3_accept(logits, gu.i32(indptr), gu.i32(proposed), top3, acc, nxt)
+    ctx = gu.i32(1000 + 10 * np.arange(len(indptr) - 1))
+    kap.top3_accept(logits, gu.i32(indptr), gu.i32(proposed), top3, acc, nxt, ctx_len=ctx)
     torch.cuda.synchronize()
+    # the commit step: every rejected proposal leaves the context
+    k = np.diff(indptr) - 1
+    np.testing.assert_array_equal(ctx.cpu().numpy(), 1000 + 10 * np.arange(len(k)) - (k - acc.cpu().numpy()))
     return top3.cpu().numpy(), acc.cpu().numpy(), nxt.cpu().numpy()
 
 
