@@ -229,9 +229,11 @@ kap_status kap_selected_decode_attn(
  * position p_j = ctx_len[b] - n_q + j and sees every token t <= p_j of the full block table
  * (ctx_len counts the rows' own tokens, whose K/V are already in the pool: the verifier advances
  * the full KV state in the same pass).  Same formula, same kernels as the proposal path.
- * bt_pages may list more pages than ceil(ctx_len / P) per sequence; only the first
- * ceil(ctx_len / P) are read.  `ws` must hold a schedule made from list_len[b] = ceil(ctx_len[b]/P)
- * and the same n_q.  Errors as kap_selected_decode_attn.
+ * bt_pages may list more pages than the schedule's list_len[b] per sequence; only the first
+ * list_len[b] are read.  `ws` must hold a schedule made with the same n_q and with
+ * list_len[b] >= ceil(ctx_len[b] / P): normally equal, but a schedule made for the longest context
+ * a graph-captured loop can reach serves every shorter one - pages at or beyond ctx_len are read
+ * (they must be valid pool pages) and contribute nothing.  Errors as kap_selected_decode_attn.
  */
 kap_status kap_verify_attn(
     const void* q,                     /* DEVICE bf16 [sum n_q, Hq, d], a sequence's rows contiguous */
