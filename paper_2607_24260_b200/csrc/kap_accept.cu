@@ -5,7 +5,8 @@
 // was not accepted (the bonus position when everything was accepted).
 //
 // Kernel 1: a cluster of up to 8 CTAs per logits row finds the row's top 3 (value descending, index ascending on
-// ties, NaN ranked below everything, -inf included) - a pure streaming reduction over the vocabulary.
+// ties, NaN ranked below everything, -inf included) - a pure streaming reduction over the vocabulary; the
+// CTAs push their candidates into the first CTA's shared memory and arrive on its mbarrier.
 // Kernel 2: one thread per sequence walks its rows.
 #include <cuda_runtime.h>
 
@@ -19,17 +20,30 @@ void count_launch();
 
 namespace {
 
-// A candidate is one 64-bit key that sorts the way the rule ranks: the logit mapped to an
-// order-preserving unsigned integer in the high word (NaN -> 0, below -inf), the complemented index
-// in the low word (lower index wins ties).  Keeping the best three is then five branch-free
-// max / min operations per logit - no divergence, whatever the data.
+// A logit is ranked by an order-preserving unsigned image of its value (NaN -> 1, below -inf,
+// which maps to 0x007fffff; 0 = "no candidate").  While a thread scans its share of the row - in
+// ascending index order - it keeps the best three images and their indices with three compares
+// and twelve selects per logit, no branches: a strictly greater image moves in, so the lower
+// index stays ahead on equal values.  For the merges between threads, warps and CTAs a candidate
+// becomes one 64-bit key (image in the high word, complemented index in the low word), and
+// keeping the best three of those is five max / min operations.
 typedef unsigned long long Key;
 struct Top3 { Key k[3]; };                                     // k[0] >= k[1] >= k[2]; 0 = empty
+struct Scan3 { uint32_t u0, u1, u2; int i0, i1, i2; };         // u0 >= u1 >= u2; 0 = empty
 
-__device__ __forceinline__ Key make_key(float v, int i) {
-    uint32_t u = __float_as_uint(v + 0.0f);                     // -0.0 and +0.0 are the same value
-    u = (v != v) ? 0u : (u ^ ((u >> 31) ? 0xffffffffu : 0x80000000u));
-    return ((Key)u << 32) | (uint32_t)~i;
+__device__ __forceinline__ uint32_t image(float v) {
+    const uint32_t u = __float_as_uint(v + 0.0f);               // -0.0 and +0.0 are the same value
+    return (v != v) ? 1u : (u ^ ((u >> 31) ? 0xffffffffu : 0x80000000u));
+}
+__device__ __forceinline__ void feed(Scan3& s, float v, int i) {
+    const uint32_t u = image(v);
+    const bool g0 = u > s.u0, g1 = u > s.u1, g2 = u > s.u2;
+    s.u2 = g1 ? s.u1 : (g2 ? u : s.u2);  s.i2 = g1 ? s.i1 : (g2 ? i : s.i2);
+    s.u1 = g0 ? s.u0 : (g1 ? u : s.u1);  s.i1 = g0 ? s.i0 : (g1 ? i : s.i1);
+    s.u0 = g0 ? u : s.u0;                s.i0 = g0 ? i : s.i0;
+}
+__device__ __forceinline__ Key as_key(uint32_t u, int i) {
+    return u ? (((Key)u << 32) | (uint32_t)~i) : 0ull;
 }
 __device__ __forceinline__ int key_index(Key k) { return (int)~(uint32_t)k; }
 __device__ __forceinline__ void push(Top3& t, Key x) {
@@ -37,43 +51,62 @@ __device__ __forceinline__ void push(Top3& t, Key x) {
     const Key b1 = max(t.k[1], r1), r2 = min(t.k[1], r1);
     t.k[0] = b0; t.k[1] = b1; t.k[2] = max(t.k[2], r2);
 }
-__device__ __forceinline__ Top3 empty_top3() { Top3 t; t.k[0] = t.k[1] = t.k[2] = 0; return t; }
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 
 // grid = rows * S CTAs in clusters of S: the S CTAs of a cluster share one row (a slice of the
 // vocabulary each) and the cluster's first CTA merges their candidates through distributed
 // shared memory.
-__global__ void __launch_bounds__(256)
+constexpr int kRowsThreads = 256;                  // 512 measured slower: fewer clusters are resident at a time
+__global__ void __launch_bounds__(kRowsThreads)
 kap_top3_rows_kernel(const float* __restrict__ logits, long long row_stride, int vocab, int S,
                      int32_t* __restrict__ top3)
 {
+    // the prefix kernel is launched programmatically behind this one: let it become resident now
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int r = blockIdx.x / S, part_id = blockIdx.x % S;
+    __shared__ unsigned long long landed;           // first CTA: completes when all peers have pushed
+    if (S > 1) {
+        if (threadIdx.x == 0 && part_id == 0) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;"
+                         ::"r"((uint32_t)__cvta_generic_to_shared(&landed)), "r"(S - 1) : "memory");
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    }
     const float* row = logits + (long long)r * row_stride;
     const int per = (vocab + S - 1) / S;
     const int lo = min(vocab, part_id * per), hi = min(vocab, lo + per);
-    Top3 t = empty_top3();
+    Scan3 sc = {0u, 0u, 0u, 0, 0, 0};
     // 16-byte loads where the slice allows it, scalar head and tail otherwise
     const int head = min(hi - lo, (int)(((16 - (reinterpret_cast<uintptr_t>(row + lo) & 15)) & 15) / 4));
-    for (int i = lo + threadIdx.x; i < lo + head; i += blockDim.x) push(t, make_key(row[i], i));
+    for (int i = lo + threadIdx.x; i < lo + head; i += blockDim.x) feed(sc, row[i], i);
     const int n4 = (hi - lo - head) / 4;
     const float4* row4 = reinterpret_cast<const float4*>(row + lo + head);
-    for (int j0 = threadIdx.x; j0 < n4; j0 += 8 * blockDim.x) {       // eight loads in flight per thread
-        float4 x[8];
+    constexpr int kInFlight = 8;                                      // loads in flight per thread
+    for (int j0 = threadIdx.x; j0 < n4; j0 += kInFlight * blockDim.x) {
+        float4 x[kInFlight];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kInFlight; ++u) {
             const int j = j0 + u * blockDim.x;
             if (j < n4) x[u] = __ldcs(row4 + j);
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kInFlight; ++u) {
             const int j = j0 + u * blockDim.x;
             if (j < n4) {
                 const int i = lo + head + 4 * j;
-                push(t, make_key(x[u].x, i)); push(t, make_key(x[u].y, i + 1));
-                push(t, make_key(x[u].z, i + 2)); push(t, make_key(x[u].w, i + 3));
+                feed(sc, x[u].x, i); feed(sc, x[u].y, i + 1);
+                feed(sc, x[u].z, i + 2); feed(sc, x[u].w, i + 3);
             }
         }
     }
-    for (int i = lo + head + 4 * n4 + threadIdx.x; i < hi; i += blockDim.x) push(t, make_key(row[i], i));
+    for (int i = lo + head + 4 * n4 + threadIdx.x; i < hi; i += blockDim.x) feed(sc, row[i], i);
+    Top3 t;
+    t.k[0] = as_key(sc.u0, sc.i0); t.k[1] = as_key(sc.u1, sc.i1); t.k[2] = as_key(sc.u2, sc.i2);
     // warp merge, then the 8 warps through shared memory
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -83,40 +116,68 @@ kap_top3_rows_kernel(const float* __restrict__ logits, long long row_stride, int
 #pragma unroll
         for (int k = 0; k < 3; ++k) push(t, o[k]);
     }
-    __shared__ Top3 part[8];
-    __shared__ Top3 cta_best;
-    __shared__ Top3 peers[8];
+    __shared__ Top3 part[kRowsThreads / 32];
+    __shared__ Top3 peers[8];                       // first CTA only: the other CTAs' candidates land here
     if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = t;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
+    // second half of the cluster barrier begun at the top: the first CTA's landing barrier is
+    // initialised and every peer is running
+    if (S > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (threadIdx.x >= 32) return;
+    // warp 0 merges the warps' candidates: lane w takes warp w's three, then a butterfly over 16 lanes
+    const int lane = threadIdx.x;
+    auto butterfly16 = [&](Top3& x) {
 #pragma unroll
-            for (int k = 0; k < 3; ++k) push(t, part[w].k[k]);
-        cta_best = t;
-    }
-    if (S > 1) {
-        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        // thread p of the first CTA fetches peer p's candidates (all peers in parallel), thread 0
-        // merges them
-        if (part_id == 0 && threadIdx.x >= 1 && threadIdx.x < S) {
-            uint32_t addr;
+        for (int off = 8; off > 0; off >>= 1) {
+            Key o[3];
+#pragma unroll
+            for (int k = 0; k < 3; ++k) o[k] = __shfl_xor_sync(0xffffffffu, x.k[k], off);
+#pragma unroll
+            for (int k = 0; k < 3; ++k) push(x, o[k]);
+        }
+    };
+    const int n_warps = (int)(blockDim.x >> 5);
+    if (lane < n_warps) t = part[lane]; else t.k[0] = t.k[1] = t.k[2] = 0;
+    butterfly16(t);                                 // lanes 0..15 now all hold the CTA's best three
+    if (S > 1 && part_id != 0) {
+        // push this CTA's three candidates into the first CTA's shared memory and arrive on its
+        // barrier (the arrive orders the stores before it); nobody reads this CTA's memory
+        if (lane == 0) {
+            uint32_t dst, bar;
             asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
-                         : "=r"(addr) : "r"((uint32_t)__cvta_generic_to_shared(&cta_best)), "r"((int)threadIdx.x));
-            Top3 o;
+                         : "=r"(dst) : "r"((uint32_t)__cvta_generic_to_shared(&peers[part_id])), "r"(0));
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+                         : "=r"(bar) : "r"((uint32_t)__cvta_generic_to_shared(&landed)), "r"(0));
 #pragma unroll
             for (int k = 0; k < 3; ++k)
-                asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(o.k[k]) : "r"(addr + 8 * k));
-            peers[threadIdx.x] = o;
+                asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(dst + 8 * k), "l"(t.k[k]) : "memory");
+            asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
         }
-        __syncthreads();
-        if (part_id == 0 && threadIdx.x == 0)
-            for (int peer = 1; peer < S; ++peer)
-#pragma unroll
-                for (int k = 0; k < 3; ++k) push(t, peers[peer].k[k]);
-        // keep every CTA's shared memory alive until the first CTA has read it
-        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        return;
     }
-    if (part_id == 0 && threadIdx.x == 0) {
+    if (S > 1) {
+        // bounded wait for the S - 1 arrivals; on a time-out the row keeps what this CTA found
+        const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&landed);
+        bool ok = false;
+        const unsigned long long give_up = global_ns() + 2000000000ull;
+        for (uint32_t spin = 0; !ok; ++spin) {
+            uint32_t done;
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], 0;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(done) : "r"(bar) : "memory");
+            ok = done != 0;
+            if (!ok && (spin & 255u) == 255u && global_ns() > give_up) break;
+        }
+        ok = __all_sync(0xffffffffu, ok);           // the lanes decide together
+        if (ok) {
+            if (lane >= 1 && lane < S) t = peers[lane];
+            else if (lane != 0) t.k[0] = t.k[1] = t.k[2] = 0;
+            butterfly16(t);                         // S <= 8 peers
+        }
+    }
+    if (lane == 0) {
 #pragma unroll
         for (int k = 0; k < 3; ++k) top3[(long long)r * 3 + k] = key_index(t.k[k]);
     }
@@ -130,6 +191,8 @@ __global__ void kap_accept_prefix_kernel(const int32_t* __restrict__ top3, const
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     const int r0 = row_indptr[b], n = row_indptr[b + 1] - r0;     // n = k + 1 rows
+    // everything above reads the caller's inputs only; top3 comes from the kernel in front
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     int m = 0;
     if (n <= 0) { accepted[b] = 0; next_token[b] = -1; return; }
     while (m < n - 1) {
@@ -175,7 +238,7 @@ extern "C" kap_status kap_top3_accept(
     attr[0].val.clusterDim.x = (unsigned)S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)total_rows * (unsigned)S);
-    cfg.blockDim = dim3(256);
+    cfg.blockDim = dim3(kRowsThreads);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = S > 1 ? 1 : 0;
@@ -183,9 +246,18 @@ extern "C" kap_status kap_top3_accept(
     cudaError_t e = cudaLaunchKernelEx(&cfg, kap_top3_rows_kernel, logits, stride, vocab, S, top3);
     if (e == cudaSuccess) {
         count_launch();
-        kap_accept_prefix_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, stream>>>(top3, row_indptr, proposed,
-                                                                                    batch, accepted, next_token, ctx_len);
-        e = cudaGetLastError();
+        cudaLaunchAttribute pa[1];
+        pa[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        pa[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t pc{};
+        pc.gridDim = dim3((unsigned)((batch + 127) / 128));
+        pc.blockDim = dim3(128);
+        pc.stream = stream;
+        pc.attrs = pa;
+        pc.numAttrs = 1;
+        const int32_t* top3_in = top3;
+        e = cudaLaunchKernelEx(&pc, kap_accept_prefix_kernel, top3_in, row_indptr, proposed, batch, accepted,
+                               next_token, ctx_len);
         if (e == cudaSuccess) count_launch();
     }
     if (e != cudaSuccess) return fail(KAP_ERR_CUDA, "kap_top3_accept launch failed: %s", cudaGetErrorString(e));
