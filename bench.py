@@ -138,6 +138,7 @@ class Cycle:
         self.pool = torch.empty((self.layers, w.num_pool_pages, 2, Hkv, P, d),
                                 dtype=torch.bfloat16, device=device)
         synth.device_fill_normal_(self.pool, 0.5, seed + 1)
+        self._plant = name == "c3"      # configuration 3: +2 sigma keys inside the selected pages
         rows_v = int(w.n_q.sum())
         self.q_dec = torch.randn((self.k, self.layers, B, Hq, d), device=device,
                                  generator=self._gen(seed + 2)).to(torch.bfloat16)
@@ -146,6 +147,11 @@ class Cycle:
         self.out_dec = torch.zeros_like(self.q_dec)
         self.out_ver = torch.zeros_like(self.q_ver)
         i32 = lambda a: torch.from_numpy(np.array(a, dtype=np.int32)).to(device)
+        if self._plant:
+            per_seq = [self.plan["plan_phys_pages"][self.plan["plan_indptr"][b]:self.plan["plan_indptr"][b + 1]]
+                       for b in range(B)]
+            for layer in range(self.layers):
+                synth.plant_affinity_keys_(self.pool[layer], self.q_dec[0, layer], w, per_seq, seed, layer)
         self.d_plan_indptr = i32(self.plan["plan_indptr"])
         self.d_plan_phys = i32(self.plan["plan_phys_pages"])
         self.d_plan_logical = i32(self.plan["plan_logical_pages"])

@@ -28,6 +28,11 @@ def _device_case(name, seed=0):
     g = torch.Generator(device=gu.DEV)
     g.manual_seed(seed + 12)
     q = torch.randn((int(w.n_q.sum()), w.num_q_heads, w.head_dim), device=gu.DEV, generator=g).to(torch.bfloat16)
+    if name == "c3":        # planted keys with a +2 sigma affinity to the decode queries, inside the plan's pages
+        plan = kap.compile_workload(w)
+        per_seq = [plan["plan_phys_pages"][plan["plan_indptr"][b]:plan["plan_indptr"][b + 1]] for b in range(w.batch)]
+        qd = q[torch.from_numpy(w.q_indptr[1:] - 1).long().to(gu.DEV)].contiguous()
+        assert synth.plant_affinity_keys_(pool, qd, w, per_seq, seed=seed, layer=0) > 0
     return w, pool, q
 
 

@@ -139,6 +139,13 @@ def test_scaled_configs(name, kwargs, peaky):
     for k in ("plan_indptr", "plan_logical_pages", "plan_phys_pages", "plan_flags", "selected_tokens"):
         np.testing.assert_array_equal(plan[k], ref_plan[k])
     qd = _decode_rows(w, q_bits)
+    if name == "c3":
+        # configuration 3 plants keys with a +2 sigma affinity to the queries inside the selected
+        # pages; the oracle gets the pool's bits back after planting
+        per_seq = [plan["plan_phys_pages"][plan["plan_indptr"][b]:plan["plan_indptr"][b + 1]] for b in range(w.batch)]
+        n = synth.plant_affinity_keys_(pool, gu.bits_to_dev(qd), w, per_seq, seed=3, layer=0, q_std=8.0)
+        assert n > 0
+        pool_bits = gu.dev_to_bits(pool)
     _check_pair(gu.run_decode(qd, pool, plan, w.ctx_len), gu.oracle_decode(qd, pool_bits, ref_plan, w.ctx_len),
                 f"{name} scaled decode")
     _check_pair(gu.run_verify(q_bits, w.n_q, pool, w.bt_indptr, w.bt_pages, w.ctx_len),
