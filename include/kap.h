@@ -376,9 +376,11 @@ kap_status kap_phase_model(double k, double h, double s, double w_main, double w
  * entry, a page outside the pool, a context that outgrew the reservation, ctx_len <= 0) set
  * 1 << KAP_ERR_DEVICE_INDEX in *device_status, or in the status word of `ws` when device_status is
  * NULL, and leave the affected entries empty (unchanged when the page of the last token itself
- * is missing).  `ws` (may be NULL) is the workspace of the
- * attention call that will read the arrays: its next launch is then issued without programmatic
- * dependent launch, because the attention prologue reads the lists ahead of the dependency wait.
+ * is missing).  `ws` is the workspace of the attention call that will read the arrays: its next
+ * launch is then issued without programmatic dependent launch, because the attention prologue
+ * reads the lists ahead of the dependency wait.  With ws == NULL that ordering is the caller's
+ * job: put another kernel between this call and the attention call, or switch programmatic
+ * dependent launch off (kap_set_launch_options).
  * Errors: KAP_ERR_UNSUPPORTED (page_size > 16), KAP_ERR_INVALID_ARG, KAP_ERR_CUDA.
  */
 kap_status kap_compile_growing_plan(
