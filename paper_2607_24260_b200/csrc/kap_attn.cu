@@ -56,6 +56,7 @@ constexpr uint64_t kWaitBudgetNs = 2000000000ull;         // per-CTA deadline fo
 // and the rest of the array as the landing zone of the push-style cluster reduction (see the
 // epilogue): C * ceil(cells / C) <= kPushCells + 16 cells of (float4 o, float2 (m, l)) each.
 constexpr int kPushIds = 256;
+constexpr int kPlainIds = 1600;                           // physical ids only: the whole array
 constexpr int kPushRows = 4;
 constexpr int kPushCells = kPushRows * 32;                // (row, 4-column) cells of the item
 constexpr int kZoneCells = kPushCells + kMaxCluster;
@@ -326,7 +327,11 @@ __device__ __forceinline__ void merge_group_cell(const AttnParams& p, const Merg
 // kNhd selects the pool layout: false = [page][2][Hkv][P][d] ("HND": a page-head's K rows are
 // contiguous; one 2-D tensor map over [rows][d]); true = [page][2][P][Hkv][d] ("NHD": token-major;
 // a 3-D tensor map (d, head, token row) whose 64 x 1 x 16 box lands in the same shared-memory tile).
-template <bool kPush, bool kNhd>
+//
+// kMode: 0 = general; 1 = push-style cluster reduction (kPush above); 2 = plain lists (kPlain: the
+// caller gave neither logical page indices nor token masks - the verification path and the
+// full-context fallback - so a CTA keeps only physical page ids and can hold 2.5 times as many).
+template <int kMode, bool kNhd>
 __global__ void __launch_bounds__(kThreads, 3)
 kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
 {
@@ -366,13 +371,14 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     const int n_item = item.page_end - item.page_begin;      // pages of the whole item
     const int slice0 = rank * (n_item / C) + min(rank, n_item % C);
     int n_local = n_item / C + (rank < n_item % C ? 1 : 0);  // pages of this CTA
-    constexpr int kIdCap = kPush ? kPushIds : kMaxIds;
+    constexpr bool kPush = kMode == 1, kPlain = kMode == 2;
+    constexpr int kIdCap = kPush ? kPushIds : kPlain ? kPlainIds : kMaxIds;
     if (n_local > kIdCap) {                                  // the scheduler caps a CTA's share at 512
         if (tid == 0) atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX);
         n_local = kIdCap;
     }
     constexpr bool push = kPush;
-    constexpr int cap = push ? kPushIds : kMaxIds;
+    constexpr int cap = kIdCap;
     if (push && (C < 2 || rows > kPushRows)) {               // the host never launches this; the
         if (tid == 0) atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX);   // landing zone would not fit
         return;                                              // (same decision in the whole cluster)
@@ -404,12 +410,12 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         // the three loads are independent of one another: one round trip
         const bool listed = (list0 + i) < list_end;
         int32_t ph = listed ? p.phys_pages[list0 + i] : -1;
-        const int32_t lg = listed && p.logical_pages ? p.logical_pages[list0 + i] : item.page_begin + i;
-        const uint16_t mk = listed && p.token_masks ? p.token_masks[list0 + i] : (uint16_t)0xFFFFu;
         if (ph < 0 || ph >= p.num_pool_pages) { ph = 0; atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX); }
         id_phys[j] = ph;
-        id_logical[j] = lg;
-        id_mask[j] = mk;
+        if (!kPlain) {
+            id_logical[j] = listed && p.logical_pages ? p.logical_pages[list0 + i] : item.page_begin + i;
+            id_mask[j] = listed && p.token_masks ? p.token_masks[list0 + i] : (uint16_t)0xFFFFu;
+        }
     }
     __syncthreads();
     // the offsets in the ring were written by ordinary stores; the bulk copies that overwrite them
@@ -464,7 +470,8 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
             const int fresh_from = L_hint - item.n_q;
             while (filled < depth) {
                 const int idx = filled * n_groups + grp;
-                if (filled >= group_pages || id_logical[idx] * kPageSize + kPageSize - 1 >= fresh_from) break;
+                const int lg = kPlain ? item.page_begin + slice0 + idx : id_logical[idx];
+                if (filled >= group_pages || lg * kPageSize + kPageSize - 1 >= fresh_from) break;
                 fill(grp * depth + filled, filled);
                 ++filled;
             }
@@ -531,10 +538,10 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         if (i == 0) KAP_TRACE_POINT(blockIdx.x, 3);
         const int page = tail->slot_page[s];
         if (page < 0 || tail->timed_out) break;              // the list is exhausted
-        const uint32_t tmask = id_mask[page];
+        const uint32_t tmask = kPlain ? 0xFFFFu : id_mask[page];
         const uint32_t kb = smem_u32(ring + s * kPageHeadBytes);
         const uint32_t vb = kb + kTileBytes;
-        const int tok0 = id_logical[page] * kPageSize;
+        const int tok0 = (kPlain ? item.page_begin + slice0 + page : id_logical[page]) * kPageSize;
 
         // S = Q K^T for the page's 16 tokens (two n-tiles of 8)
         float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -880,8 +887,9 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     if (st != KAP_OK) return st;
     // function attributes are per device: set them once for the workspace's device
     if (!ws->attrs_set) {
-        const void* variants[4] = {(const void*)kap_attn_split_kernel<false, false>, (const void*)kap_attn_split_kernel<true, false>,
-                                   (const void*)kap_attn_split_kernel<false, true>, (const void*)kap_attn_split_kernel<true, true>};
+        const void* variants[6] = {(const void*)kap_attn_split_kernel<0, false>, (const void*)kap_attn_split_kernel<1, false>,
+                                   (const void*)kap_attn_split_kernel<2, false>, (const void*)kap_attn_split_kernel<0, true>,
+                                   (const void*)kap_attn_split_kernel<1, true>, (const void*)kap_attn_split_kernel<2, true>};
         for (const void* fn : variants) {
             cudaError_t ae = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_for(kMaxSlots));
             if (ae != cudaSuccess) return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ae));
@@ -927,10 +935,17 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     // few rows and short lists in every item (the proposal path): push-style cluster reduction
     const bool push = ws->cluster_size > 1 && ws->max_nq * p.G <= kPushRows && ws->max_chunk <= kPushIds;
     const bool nhd = ws->kv_layout == KAP_KV_NHD;
-    if (push && nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<true, true>, *map, p));
-    else if (push) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<true, false>, *map, p));
-    else if (nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<false, true>, *map, p));
-    else KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<false, false>, *map, p));
+    // neither logical indices nor masks: physical ids only (longer slices fit a CTA)
+    const bool plain = !push && !p.logical_pages && !p.token_masks;
+    if (!plain && !push && ws->max_chunk > kMaxIds)
+        return fail(KAP_ERR_INVALID_ARG, "the schedule's slices of %d pages need plain page lists (no logical "
+                    "indices, no masks)", ws->max_chunk);
+    if (push && nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<1, true>, *map, p));
+    else if (push) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<1, false>, *map, p));
+    else if (plain && nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<2, true>, *map, p));
+    else if (plain) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<2, false>, *map, p));
+    else if (nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<0, true>, *map, p));
+    else KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<0, false>, *map, p));
     g_launches.fetch_add(1);
     if (ws->n_merge_groups > 0) {
         const int rows = ws->max_nq * p.G;
@@ -1045,10 +1060,10 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     KAP_CUDA(cudaSetDevice(ws->device));
     const int ring_slots = g_ring_slots.load();
     const int smem = smem_bytes_for(ring_slots);
-    cudaFuncSetAttribute(kap_attn_split_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(kap_attn_split_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          smem_bytes_for(kMaxSlots));
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel<false, false>, kThreads, smem) != cudaSuccess || occ < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel<0, false>, kThreads, smem) != cudaSuccess || occ < 1)
         occ = 1;
     const int want = g_ctas_per_sm.load();
     const int per_sm = want > 0 ? std::min(want, occ) : occ;
@@ -1056,7 +1071,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     ws->ring_slots = ring_slots;
     ws->ctas_per_wave = per_sm * ws->sm_count;
     int32_t slots[kMaxCluster] = {ws->ctas_per_wave};
-    cudaFuncSetAttribute(kap_attn_split_kernel<false, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    cudaFuncSetAttribute(kap_attn_split_kernel<0, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     cudaGetLastError();
     for (int c = 2; c <= kMaxCluster; ++c) {
         if (c > g_max_cluster.load()) continue;
@@ -1069,7 +1084,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         cc.dynamicSmemBytes = smem;
         cc.attrs = ca; cc.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel<false, false>, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
+        if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel<0, false>, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
         slots[c - 1] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
     }
     // A one-wave schedule of the proposal path leaves a third of the SM's CTA slots to the next
@@ -1329,7 +1344,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
         if (!g_static_ready[dev]) {
             void* ptr = nullptr;
             KAP_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
-            KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel<false, false>,
+            KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel<0, false>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           smem_bytes_for(kMaxSlots)));
             g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
@@ -1384,7 +1399,7 @@ extern "C" kap_status kap_selected_decode_attn_static(
     g_launches.fetch_add(1);
     // plain launches: the work list was written by the kernel just before, so the split kernel
     // must not start early
-    kap_attn_split_kernel<false, false><<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
+    kap_attn_split_kernel<0, false><<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
     KAP_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     if (num_splits > 1) {

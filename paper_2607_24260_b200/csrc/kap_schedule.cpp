@@ -38,7 +38,8 @@ constexpr int64_t kMergePassPages = 9;
 constexpr int64_t kLaterWavePages = 40;
 constexpr int64_t kClusterPagesX5 = 8;                    // per CTA of a cluster, in fifths of a page
 constexpr int64_t kPushClusterPagesX5 = 4;                // same, when the kernel reduces by pushing (<= 4 rows)
-constexpr int32_t kDefaultChunkCap = 512;     // per CTA; also the size of the kernel's page-id buffer
+constexpr int32_t kDefaultChunkCap = 512;     // pages per CTA: the kernel's page-id buffer holds 640 entries
+constexpr int32_t kPlainChunkCap = 1536;      // verification lists carry physical ids only: 1600 fit
 
 // cluster_slots[c - 1] = clusters of c CTAs that can be resident at once (0 = size not allowed);
 // one_wave_slots[c - 1] = how many of them a schedule that fits one wave may use: leaving part of
@@ -56,7 +57,8 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
     const int32_t G = num_q_heads / num_kv_heads;
     if (kRowTile % G) return fail(KAP_ERR_UNSUPPORTED, "group size %d must divide %d", G, kRowTile);
     if (cluster_slots[0] <= 0) return fail(KAP_ERR_INVALID_ARG, "cta_slots %d", cluster_slots[0]);
-    const int32_t cap = max_chunk_pages <= 0 ? kDefaultChunkCap : std::min(max_chunk_pages, kDefaultChunkCap);
+    const int32_t hard_cap = n_q ? kPlainChunkCap : kDefaultChunkCap;
+    const int32_t cap = max_chunk_pages <= 0 ? hard_cap : std::min(max_chunk_pages, hard_cap);
     int32_t max_len = 0, max_nq = 1;
     for (int32_t b = 0; b < batch; ++b) {
         if (list_len[b] <= 0) return fail(KAP_ERR_INVALID_ARG, "list_len[%d] = %d <= 0", b, list_len[b]);

@@ -7,6 +7,9 @@ import pytest
 from paper_2607_24260_b200 import kap, synth
 
 
+PROPOSAL_CAP, VERIFY_CAP = 512, 1536      # pages per CTA: plan lists (ids + logical + masks) / plain lists
+
+
 def _verify_schedule(list_len, n_q, items, Hkv, cap, cluster=1):
     B = len(list_len)
     cover = [[np.zeros(int(list_len[b]), dtype=np.int32) for _ in range(Hkv)] for b in range(B)]
@@ -54,7 +57,7 @@ def test_named_configs_schedules(name):
         assert feasible(max_chunk) and not feasible(max_chunk - 1)
     pages = (w.ctx_len + 15) // 16
     items, n_merge, max_chunk = kap.schedule_host(pages, w.n_q, 32, 8, slots)
-    _verify_schedule(pages, w.n_q, items, 8, 512)
+    _verify_schedule(pages, w.n_q, items, 8, VERIFY_CAP)
 
 
 def test_random_shapes_and_caps():
@@ -67,7 +70,8 @@ def test_random_shapes_and_caps():
         cap = int(rng.choice([0, 1, 3, 64, 512, 100000]))
         slots = int(rng.choice([4, 148, 296]))
         items, _, _ = kap.schedule_host(n, nq, Hkv * 4, Hkv, slots, cap, max_items=200000)
-        _verify_schedule(n, nq, items, Hkv, 512 if cap <= 0 else min(cap, 512))
+        hard = PROPOSAL_CAP if nq is None else VERIFY_CAP
+        _verify_schedule(n, nq, items, Hkv, hard if cap <= 0 else min(cap, hard))
 
 
 def test_single_wave_is_minimal_makespan():
@@ -113,4 +117,4 @@ def test_cluster_schedules():
         items, n_merge, max_chunk, cluster = kap.schedule_host(n, nq, 32, 8, int(rng.choice([296, 444])),
                                                                max_items=100000, max_cluster=mc)
         assert 1 <= cluster <= mc
-        _verify_schedule(n, nq, items, 8, 512, cluster)
+        _verify_schedule(n, nq, items, 8, PROPOSAL_CAP if nq is None else VERIFY_CAP, cluster)
