@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read+write per launch / algorithmic bytes per launch, from the ncu captures
 # summarised under profiles/kap_attn_split_kernel_c2_c3_c4.md (c2 captured with 4 of its 32 layers;
 # traffic per launch does not depend on the layer count)
-TRAFFIC_RATIO = {"decode": 1.011, "verify": 1.008}
+TRAFFIC_RATIO = {"decode": 1.018, "verify": 1.007}
 
 
 def measured_peak():
