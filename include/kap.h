@@ -508,9 +508,12 @@ kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);
  *   early_kv     != 0 (default; needs use_pdl): in that window the kernel also reads ctx_len as a
  *                hint and starts loading KV pages that hold only tokens older than the query
  *                rows' own (t < ctx_len - n_q) - pages written in earlier decoding steps.  Those
- *                pages must then be final before the previous kernel was launched, and ctx_len may
- *                only grow while it runs (the masks use the value read after the wait); Q, the
- *                pages holding the rows' own tokens, out and lse may still be written by it.
+ *                pages must then be final before the previous kernel was launched; ctx_len may be
+ *                advanced by it by at most n_q, or lowered (the masks use the value read after
+ *                the wait); Q, the pages holding the rows' own tokens, out and lse may still be
+ *                written by it.  kap_append_kv with several new tokens per sequence (new_indptr
+ *                given) could break the first condition for the call that follows it, so the
+ *                library starts that one attention launch's loads after the wait.
  *   ctas_per_sm  resident CTAs per SM the scheduler fills in one wave; 0 = as many as fit.
  *   max_cluster  largest thread-block cluster (1 .. 16; default 16, sizes above 8 use the
  *                non-portable cluster launch) the scheduler may give a work item.  The CTAs of a cluster share the item's pages and reduce their partial

@@ -11,6 +11,7 @@
 
 namespace kap {
 void count_launch();
+void kv_written_in_bulk();
 
 namespace {
 
@@ -81,5 +82,8 @@ extern "C" kap_status kap_append_kv(
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(KAP_ERR_CUDA, "kap_append_kv launch failed: %s", cudaGetErrorString(e));
     count_launch();
+    // with several new tokens per sequence the next attention kernel's early page loads could
+    // touch tokens this kernel is still writing: that launch starts its loads after the wait
+    if (new_indptr) kv_written_in_bulk();
     return KAP_OK;
 }

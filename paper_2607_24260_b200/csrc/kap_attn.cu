@@ -460,7 +460,8 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     // Early KV prefetch: pages that hold only tokens older than the query rows' own tokens
     // (t < L - n_q) were written in earlier steps, so their loads may start before the previous
     // kernel on the stream has completed.  Pages holding the rows' own tokens, Q and the partial
-    // buffers wait for it.  (ctx_len may only grow while the previous kernel runs.)
+    // buffers wait for it.  (What the previous kernel may do to ctx_len: advance it by at most n_q,
+    // or lower it - a lowered value only means that some prefetched pages end up masked.)
     int filled = 0;
     if (p.early_kv) {
         // a hint only: if the previous kernel is still advancing ctx_len, an older (smaller) value
@@ -795,6 +796,10 @@ std::atomic<long long> g_launches{0};
 void count_launch() { g_launches.fetch_add(1); }       // for the library's other translation units
 int32_t* workspace_status_word(kap_workspace* ws) { return ws->d_status; }
 void workspace_lists_rewritten(kap_workspace* ws) { ws->plain_next = 1; }
+namespace { std::atomic<int> g_no_early_once{0}; }
+// a kernel that wrote several tokens per sequence into the KV pool was just enqueued: the next
+// attention launch must not start loading "older" pages before that kernel has completed
+void kv_written_in_bulk() { g_no_early_once.store(1); }
 namespace {
 
 std::atomic<int> g_use_pdl{1};
@@ -906,7 +911,7 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     // the dependency wait) must not overlap the writer: one ordinary launch, then back to normal
     const bool use_pdl = g_use_pdl.load() && !ws->plain_next;
     ws->plain_next = 0;
-    p.early_kv = (use_pdl && g_early_kv.load()) ? 1 : 0;
+    p.early_kv = (use_pdl && g_early_kv.load() && !g_no_early_once.exchange(0)) ? 1 : 0;
 #ifdef KAP_TRACE
     p.trace = (g_trace && g_trace_next < g_trace_cap) ? g_trace + (size_t)(g_trace_next++) * 8192 * 8 : nullptr;
 #endif

@@ -114,3 +114,46 @@ def test_append_reports_missing_page():
     torch.cuda.synchronize()
     assert int(status.item()) == 1 << kap.ERR_DEVICE_INDEX
     np.testing.assert_array_equal(gu.dev_to_bits(pool), pool_bits)     # nothing was written
+
+
+def test_bulk_append_then_decode_sees_every_new_token():
+    """Several tokens per sequence appended by one call, the proposal-path attention enqueued right
+    behind it on the same stream (programmatic dependent launch on): the attention must see all
+    of them - its early page loads may not run ahead of the append."""
+    w, end = _cycle_case(5, 7, (1000, 2040, 333))
+    B, Hq, Hkv, d = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim
+    rng = synth.rng_for(5, "bulk-append")
+    n_new = np.array([7, 3, 5], dtype=np.int32)
+    indptr = np.concatenate([[0], np.cumsum(n_new)]).astype(np.int32)
+    q_bits, pool_bits = synth.host_qkv(w, 5, q_rows=B, q_std=4.0)
+    k_new = synth.normal_bf16((int(n_new.sum()), Hkv, d), 0.5, rng)
+    v_new = synth.normal_bf16((int(n_new.sum()), Hkv, d), 0.5, rng)
+    final = (w.ctx_len + n_new).astype(np.int32)
+    plan = kap.compile_plan(final, w.span_indptr, w.span_start, w.span_len, w.span_score,
+                            w.budget_tokens + 7, w.n_sink, w.n_recent + 7, None, 1.0, w.bt_indptr, w.bt_pages)
+    pool = gu.bits_to_dev(pool_bits)
+    d_ctx = gu.i32(w.ctx_len)
+    d_q = gu.bits_to_dev(q_bits)
+    d_out = torch.zeros_like(d_q)
+    ws = kap.Workspace(max_rows_per_item=Hq // Hkv, max_batch=B)
+    ws.schedule(np.diff(plan["plan_indptr"]), None, Hq, Hkv)
+    args = (gu.i32(plan["plan_indptr"]), gu.i32(plan["plan_phys_pages"]), gu.i32(plan["plan_logical_pages"]))
+    d_k, d_v, d_ind = gu.bits_to_dev(k_new), gu.bits_to_dev(v_new), gu.i32(indptr)
+    d_bt_indptr, d_bt_pages = gu.i32(w.bt_indptr), gu.i32(w.bt_pages)
+    for _ in range(3):                                      # repeat: a race would be intermittent
+        pool.copy_(gu.bits_to_dev(pool_bits))
+        d_ctx.copy_(gu.i32(w.ctx_len))
+        kap.selected_decode_attn(d_q, pool, *args, d_ctx, d_out, ws)          # keeps the GPU busy in front
+        kap.append_kv(d_k, d_v, pool, d_bt_indptr, d_bt_pages, d_ctx, new_indptr=d_ind, advance=True)
+        kap.selected_decode_attn(d_q, pool, *args, d_ctx, d_out, ws)
+        torch.cuda.synchronize()
+        ws.check()
+        host_pool = pool_bits.copy()
+        for b in range(B):
+            bt = w.bt_pages[w.bt_indptr[b]:w.bt_indptr[b + 1]]
+            brute.append_kv(host_pool, bt, int(w.ctx_len[b]), k_new[indptr[b]:indptr[b + 1]], v_new[indptr[b]:indptr[b + 1]])
+        ref, _, _, _ = orc.selected_decode_attn(q_bits, host_pool, plan["plan_indptr"], plan["plan_phys_pages"],
+                                                plan["plan_logical_pages"], final)
+        assert_close(gu.dev_bf16_to_f64(d_out), ref, what="decode after a bulk append")
+        np.testing.assert_array_equal(d_ctx.cpu().numpy(), final)
+    ws.close()
