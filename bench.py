@@ -553,8 +553,14 @@ def config_dict(w, k, layers, extra=None):
     c = {"workload": f"{w.name}: {w.note}", "batch": w.batch, "ctx_len_max": int(w.ctx_len.max()),
          "ctx_len_min": int(w.ctx_len.min()), "layers": layers, "proposals_per_cycle_k": k,
          "verify_rows": k, "heads": f"{w.num_q_heads}q/{w.num_kv_heads}kv", "head_dim": w.head_dim,
-         "page_size": w.page_size,
-         "l2": "no flush: every layer has its own KV slice, per-cycle working set >> 126 MB L2"}
+         "page_size": w.page_size}
+    kv_bytes = layers * int(sum((int(L) + w.page_size - 1) // w.page_size for L in w.ctx_len)) * w.page_bytes
+    c["kv_bytes_per_cycle"] = kv_bytes
+    if kv_bytes > 4 * 126e6:
+        c["l2"] = "no flush: every layer has its own KV slice, per-cycle working set >> 126 MB L2"
+    else:
+        c["l2"] = ("small case, no flush: the KV of the whole cycle fits the 126 MB L2, so its figures "
+                   "are L2-resident and say nothing about HBM bandwidth")
     if extra:
         c.update(extra)
     return c
