@@ -8,7 +8,7 @@ when the CTAs entered, finished staging their page ids, passed the dependency wa
 first page, left the main loop and ended - all in microseconds of the GPU's global timer, relative
 to the end of the previous layer.  The timestamps themselves cost about 1 us per layer.
 
-Trace slots written by thread 0 of every CTA (see KAP_TRACE_POINT in csrc/kap_attn.cu):
+Trace slots written by thread 0 of every CTA (see KAP_TRACE_POINT in csrc/kap_attn_kernel.cuh):
 0 entry, 1 page ids staged, 2 dependency wait passed, 3 first page arrived, 4 main loop left,
 6 warps combined, 5 end; slot 7 holds the SM id.
 """
