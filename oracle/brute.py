@@ -102,7 +102,9 @@ def top3_accept(logits, row_indptr, proposed):
     """Tolerant acceptance (Section 3.2, Eq. 2 with the Top-3 rule): per row the three best
     candidates (value descending, lower index first on ties, NaN below every number, -inf included); m = number of
     proposed tokens accepted consecutively from the start of each sequence's window; next carry =
-    the best candidate of row m.  logits float32 [rows, V].  Returns (top3, accepted, next)."""
+    the best candidate of row m.  A window without any row (row_indptr[b+1] == row_indptr[b]) has
+    nothing to accept and no row to take a carry from: accepted = 0, next = -1.
+    logits float32 [rows, V].  Returns (top3, accepted, next)."""
     x = np.asarray(logits, dtype=np.float32)
     rows, V = x.shape
     nan = np.isnan(x)
@@ -117,6 +119,9 @@ def top3_accept(logits, row_indptr, proposed):
     nxt = np.zeros(B, dtype=np.int32)
     for b in range(B):
         r0, n = int(row_indptr[b]), int(row_indptr[b + 1] - row_indptr[b])
+        if n <= 0:
+            accepted[b], nxt[b] = 0, -1
+            continue
         m = 0
         while m < n - 1 and int(proposed[r0 + m]) in top3[r0 + m].tolist():
             m += 1

@@ -471,6 +471,83 @@ def test_append_then_attend_equals_attention_over_the_longer_context():
         assert np.all(nv == L)
 
 
+def test_append_kv_writes_exactly_the_slot_the_mapping_names():
+    """Slot mapping by direct indexing (Section 3.1: token at logical position pos lives in page
+    block_table[pos // P], slot pos % P): after one append of a K row and a different V row, exactly
+    those two (page, K|V, :, slot) strips changed, they hold K and V respectively, and every other
+    word of the pool is untouched.  Crosses a page boundary (L % 16 in {0, 15}) and appends
+    several tokens at once."""
+    c = _small_case(21, L=95, n_q=1, spare=6)
+    free = [p for p in range(c["pool"].shape[0]) if p not in set(c["bt"].tolist())]
+    bt = np.concatenate([c["bt"], np.asarray(free[:2], dtype=np.int32)])
+    for L, n_new in ((95, 1), (96, 1), (90, 3), (94, 5)):
+        k_new = np.empty((n_new, c["Hkv"], c["d"]), dtype=np.uint16)
+        v_new = np.empty_like(k_new)
+        for j in range(n_new):                   # distinctive words no random bf16 draw produces
+            k_new[j] = 0x4100 + 2 * j + np.arange(c["Hkv"])[:, None] * 16
+            v_new[j] = 0xC200 + 2 * j + np.arange(c["Hkv"])[:, None] * 16 + 1
+        before = c["pool"].copy()
+        pool = c["pool"].copy()
+        assert brute.append_kv(pool, bt, L, k_new, v_new) == L + n_new
+        changed = np.zeros(pool.shape, dtype=bool)
+        for j in range(n_new):
+            pos = L + j
+            page, slot = int(bt[pos // P]), pos % P
+            np.testing.assert_array_equal(pool[page, 0, :, slot, :], k_new[j])
+            np.testing.assert_array_equal(pool[page, 1, :, slot, :], v_new[j])
+            changed[page, :, :, slot, :] = True
+        np.testing.assert_array_equal(pool[~changed], before[~changed])
+        assert changed.sum() == n_new * 2 * c["Hkv"] * c["d"]
+
+
+@pytest.mark.parametrize("L", [95, 96, 111, 112])
+def test_append_kv_then_decode_returns_the_appended_value(L):
+    """Closed form through the C oracle: append a key that dominates the softmax (scaled logit 60)
+    together with a known value row; full-context decode at L + 1 must return that value row for
+    the planted head.  A K/V swap, a wrong slot or a wrong page fails it."""
+    c = _small_case(22, L=L, n_q=1, spare=6)
+    free = [p for p in range(c["pool"].shape[0]) if p not in set(c["bt"].tolist())]
+    bt = np.concatenate([c["bt"], np.asarray(free[:1], dtype=np.int32)])
+    head, G = 3, c["Hq"] // c["Hkv"]
+    q = synth.bf16_bits_to_f64(c["q"][-1][head])
+    k_row = synth.normal_bf16((1, c["Hkv"], c["d"]), 0.5, c["rng"])
+    k_row[0, head // G] = synth.f32_to_bf16_bits((q * (60.0 * np.sqrt(c["d"]) / (q @ q))).astype(np.float32))
+    v_row = synth.f32_to_bf16_bits(np.linspace(-3.0, 3.0, c["Hkv"] * c["d"], dtype=np.float32)
+                                   ).reshape(1, c["Hkv"], c["d"])
+    pool = c["pool"].copy()
+    L1 = brute.append_kv(pool, bt, L, k_row, v_row)
+    assert L1 == L + 1
+    n_pages = (L1 + P - 1) // P
+    logical = np.arange(n_pages, dtype=np.int32)
+    out, lse, _, nv = orc.selected_decode_attn(c["q"][-1:], pool, [0, n_pages], bt[logical], logical, [L1])
+    np.testing.assert_allclose(out[0, head], synth.bf16_bits_to_f64(v_row[0, head // G]), atol=1e-9)
+    assert abs(lse[0, head] - 60.0) < 0.5 and np.all(nv == L1)
+    # one token short of the append the key is not there yet
+    out0, lse0, _, _ = orc.selected_decode_attn(c["q"][-1:], pool, [0, (L + P - 1) // P],
+                                                bt[:(L + P - 1) // P], logical[:(L + P - 1) // P], [L])
+    assert lse0[0, head] < 30.0
+
+
+def test_materialize_view_hand_worked():
+    """The compact copy on a pool worked by hand: five pages, page p filled with the constant
+    100 + p, plan [3, 0, 3] -> compact pages hold 103, 100, 103 and are numbered 0, 1, 2; the
+    source pool is not modified and the copy does not alias it."""
+    pool = np.empty((5, 2, 2, P, 4), dtype=np.uint16)
+    for p in range(5):
+        pool[p] = 100 + p
+    pool[3, 1] = 203                              # V half of page 3 differs from its K half
+    keep = pool.copy()
+    compact, ids = brute.materialize_view(pool, [3, 0, 3])
+    assert compact.shape == (3, 2, 2, P, 4) and ids.tolist() == [0, 1, 2]
+    assert np.all(compact[0, 0] == 103) and np.all(compact[0, 1] == 203)
+    assert np.all(compact[1] == 100)
+    assert np.all(compact[2, 0] == 103) and np.all(compact[2, 1] == 203)
+    compact[0] = 7
+    np.testing.assert_array_equal(pool, keep)
+    empty, ids0 = brute.materialize_view(pool, [])
+    assert empty.shape[0] == 0 and len(ids0) == 0
+
+
 # --------------------------------------------------------------------------- Top-3 acceptance
 def test_top3_accept_hand_cases():
     """Eq. 2 with the Top-3 rule on a window worked by hand (k = 3, vocab 6)."""
@@ -507,6 +584,17 @@ def test_top3_matches_argsort_and_prefix_definition():
     prop = top3[:, 1].copy()
     _, m, nxt = brute.top3_accept(x, indptr, prop)
     assert m.tolist() == [4, 0, 6] and nxt[0] == top3[4, 0] and nxt[2] == top3[11, 0]
+    assert nxt[1] == -1                          # a window without rows has no carry to give
     prop[6] = int(np.argsort(x[6])[0])           # the worst token at the 2nd position of window 3 (rows 5..11)
     _, m, nxt = brute.top3_accept(x, indptr, prop)
     assert m.tolist() == [4, 0, 1] and nxt[2] == top3[6, 0]
+
+
+def test_top3_empty_windows_accept_nothing_and_carry_minus_one():
+    """A window with no row at all - first, in the middle, last - yields accepted = 0 and
+    next = -1 and never reads a neighbour's row."""
+    x = np.zeros((3, 8), dtype=np.float32)
+    x[0, 5] = x[1, 6] = x[2, 7] = 1.0
+    top3, m, nxt = brute.top3_accept(x, [0, 0, 2, 2, 3, 3], [5, 0, 0])
+    assert m.tolist() == [0, 1, 0, 0, 0]
+    assert nxt.tolist() == [-1, 6, -1, 7, -1]
