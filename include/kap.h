@@ -145,9 +145,14 @@ kap_status kap_compile_plan(
  * repeats the previous call's counts and options returns at once and uploads nothing.
  * A workspace serves one attention call at a time: use one for the proposal path and another for
  * the verification path.  max_chunk_pages = 0 picks the default chunk cap.
- * Errors: KAP_ERR_INVALID_ARG (NULL, batch < 0 or > max_batch, list_len <= 0, n_q < 1, bad head
- * counts), KAP_ERR_CAPACITY (rows or items beyond what the workspace was created for),
- * KAP_ERR_CUDA.
+ * Errors: KAP_ERR_INVALID_ARG (NULL, batch < 0, list_len <= 0, n_q < 1, bad head counts),
+ * KAP_ERR_CAPACITY (batch > max_batch; rows or items beyond what the workspace was created for;
+ * max_batch > 8191: every CTA stages the batch's offset arrays in shared memory), KAP_ERR_CUDA.
+ * A kap_schedule that fails leaves the previous schedule in force, whole.
+ * Neither call changes the calling thread's current device (it is switched to the workspace's
+ * device inside the call and put back).  The attention calls, by contrast, must be made with the
+ * workspace's device current - like any launch on one of its streams - and return
+ * KAP_ERR_INVALID_ARG otherwise.
  */
 typedef struct kap_workspace kap_workspace;
 
@@ -302,6 +307,9 @@ kap_status kap_append_kv(
  *                  during the cycle, ctx_len counts all k_b of them on entry and only the accepted
  *                  ones on return; the rejected tokens' slots are overwritten by the next
  *                  cycle's appends.  The carry token is not in the cache yet.
+ * A window without any row (row_indptr[b+1] == row_indptr[b]: a sequence that sits this cycle out)
+ * has nothing to accept and no row to take a carry from: accepted[b] = 0, next_token[b] = -1,
+ * ctx_len[b] unchanged.
  * logits: DEVICE fp32, row r starts at logits + r * row_stride.  All outputs DEVICE int32; top3 is
  * [total_rows, 3] and is required (it is also the scratch between the two kernels).
  * Errors: KAP_ERR_INVALID_ARG (NULL pointer, vocab < 3, row_stride < vocab, negative counts),
@@ -462,6 +470,14 @@ kap_status kap_materialize_view(
  *   - sizes the array cannot hold are refused: batch * num_kv_heads * num_splits work items need
  *     about 32 + (Hq/Hkv) * 520 bytes each; beyond 4 MiB in total the call returns
  *     KAP_ERR_CAPACITY and enqueues nothing (with 32/8 heads: roughly 1900 work items).
+ *   - one slice (ceil(list pages / num_splits) pages of one sequence) is run by one CTA, which can
+ *     hold 640 page ids, or 1600 when plan_logical_pages is NULL.  The list lengths are on the
+ *     device, so the host cannot refuse a longer slice up front: the device cuts it to the limit,
+ *     sets 1 << KAP_ERR_CAPACITY in the status word and the output of that sequence is NOT valid
+ *     (the pages beyond the cut were not attended to).  A caller that passes device_status == NULL
+ *     gets no signal at all, so choose num_splits >= ceil(longest list / 640) (or / 1600): a
+ *     full-context list of 131 072 tokens (8192 pages) needs 13 splits with logical indices,
+ *     6 without.
  *   - all calls on a device share the array and it keeps the previous call's contents.  The call
  *     itself clears the only part that must start at zero (the status word) and rewrites the
  *     rest before use, so back-to-back calls on ONE stream are fine; calls that may overlap on
@@ -473,9 +489,10 @@ kap_status kap_materialize_view(
  *     the token-major layout belong to the workspace entry point.
  * Results are the same as the workspace entry point's up to the order of the fp32 sums.
  * device_status (DEVICE int32, may be NULL) receives the kernels' status bits after the call's
- * kernels: 0, or 1 << KAP_ERR_DEVICE_INDEX / 1 << KAP_ERR_TIMEOUT.
+ * kernels: 0, or a bit-or of 1 << KAP_ERR_DEVICE_INDEX (a page id outside the pool), 1 <<
+ * KAP_ERR_TIMEOUT and 1 << KAP_ERR_CAPACITY (a slice was cut, see above).
  * Errors: KAP_ERR_UNSUPPORTED (shape), KAP_ERR_INVALID_ARG (NULL pointer, num_splits < 1,
- * misaligned pool), KAP_ERR_CAPACITY (see above), KAP_ERR_CUDA.
+ * misaligned pool), KAP_ERR_CAPACITY (scratch size, or batch > 16 383), KAP_ERR_CUDA.
  */
 kap_status kap_selected_decode_attn_static(
     const void* q,                     /* DEVICE bf16 [batch, Hq, d] */
@@ -508,12 +525,14 @@ kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);
  *   early_kv     != 0 (default; needs use_pdl): in that window the kernel also reads ctx_len as a
  *                hint and starts loading KV pages that hold only tokens older than the query
  *                rows' own (t < ctx_len - n_q) - pages written in earlier decoding steps.  Those
- *                pages must then be final before the previous kernel was launched; ctx_len may be
- *                advanced by it by at most n_q, or lowered (the masks use the value read after
- *                the wait); Q, the pages holding the rows' own tokens, out and lse may still be
- *                written by it.  kap_append_kv with several new tokens per sequence (new_indptr
- *                given) could break the first condition for the call that follows it, so the
- *                library starts that one attention launch's loads after the wait.
+ *                pages must then be final under the same rule; ctx_len may be advanced by the
+ *                kernels still running by at most n_q, or lowered (the masks use the value read
+ *                after the wait); Q, the pages holding the rows' own tokens, out and lse may still
+ *                be written by them.  kap_append_kv with several new tokens per sequence
+ *                (new_indptr given) could break the first condition for the attention call that
+ *                follows it ON THE SAME STREAM, so the library starts that one launch's loads after
+ *                the wait; the bookkeeping is per stream, attention calls on other streams neither
+ *                lose their early loads nor use the mark up.
  *   ctas_per_sm  resident CTAs per SM the scheduler fills in one wave; 0 = as many as fit.
  *   max_cluster  largest thread-block cluster (1 .. 16; default 16, sizes above 8 use the
  *                non-portable cluster launch) the scheduler may give a work item.  The CTAs of a cluster share the item's pages and reduce their partial

@@ -11,7 +11,7 @@
 
 namespace kap {
 void count_launch();
-void kv_written_in_bulk();
+void kv_written_in_bulk(void* cuda_stream);
 
 namespace {
 
@@ -82,8 +82,9 @@ extern "C" kap_status kap_append_kv(
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(KAP_ERR_CUDA, "kap_append_kv launch failed: %s", cudaGetErrorString(e));
     count_launch();
-    // with several new tokens per sequence the next attention kernel's early page loads could
-    // touch tokens this kernel is still writing: that launch starts its loads after the wait
-    if (new_indptr) kv_written_in_bulk();
+    // with several new tokens per sequence the early page loads of the next attention kernel on
+    // this stream could touch tokens this kernel is still writing: that launch starts its loads
+    // after the dependency wait
+    if (new_indptr) kv_written_in_bulk(cuda_stream);
     return KAP_OK;
 }

@@ -30,10 +30,43 @@ std::atomic<long long> g_launches{0};
 void count_launch() { g_launches.fetch_add(1); }       // for the library's other translation units
 int32_t* workspace_status_word(kap_workspace* ws) { return ws->d_status; }
 void workspace_lists_rewritten(kap_workspace* ws) { ws->plain_next = 1; }
-namespace { std::atomic<int> g_no_early_once{0}; }
-// a kernel that wrote several tokens per sequence into the KV pool was just enqueued: the next
-// attention launch must not start loading "older" pages before that kernel has completed
-void kv_written_in_bulk() { g_no_early_once.store(1); }
+// A kernel that wrote several tokens per sequence into the KV pool was just enqueued on `stream`:
+// the next attention launch ON THAT STREAM must not start loading "older" pages before that kernel
+// has completed.  (Programmatic dependent launch only ever overlaps kernels of one stream; a launch
+// on another stream is ordered against the writer by an event, i.e. completely.)  The marks are kept
+// per stream so that a launch on another stream, workspace or thread cannot use one up.  When the
+// small table is full, every workspace's next launch is held back once instead - never less
+// cautious than needed.
+namespace {
+std::mutex g_bulk_mutex;
+constexpr int kBulkMarks = 32;
+cudaStream_t g_bulk_stream[kBulkMarks];
+int g_bulk_count = 0;
+unsigned long long g_bulk_overflows = 0;      // times the table was full
+}
+void kv_written_in_bulk(void* cuda_stream) {
+    std::lock_guard<std::mutex> lock(g_bulk_mutex);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    for (int i = 0; i < g_bulk_count; ++i)
+        if (g_bulk_stream[i] == st) return;
+    if (g_bulk_count < kBulkMarks) g_bulk_stream[g_bulk_count++] = st;
+    else ++g_bulk_overflows;
+}
+namespace {
+// true when the launch about to be enqueued on `st` follows such a write; uses the mark up
+bool take_bulk_mark(kap_workspace* ws, cudaStream_t st) {
+    std::lock_guard<std::mutex> lock(g_bulk_mutex);
+    bool marked = ws->bulk_overflows_seen != g_bulk_overflows;
+    ws->bulk_overflows_seen = g_bulk_overflows;
+    for (int i = 0; i < g_bulk_count; ++i)
+        if (g_bulk_stream[i] == st) {
+            g_bulk_stream[i] = g_bulk_stream[--g_bulk_count];
+            marked = true;
+            break;
+        }
+    return marked;
+}
+}
 namespace {
 
 std::atomic<int> g_use_pdl{1};
@@ -57,6 +90,25 @@ EncodeTiledFn encode_tiled_fn() {
         return reinterpret_cast<EncodeTiledFn>(f);
     }();
     return fn;
+}
+
+// Makes `device` current for the enclosing scope and puts the caller's device back afterwards.
+struct DeviceScope {
+    int prev = -1;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceScope(int device) {
+        err = cudaGetDevice(&prev);
+        if (err != cudaSuccess) { prev = -1; return; }
+        if (prev == device) prev = -1;            // nothing to put back
+        else err = cudaSetDevice(device);
+    }
+    ~DeviceScope() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// The prologue of the split kernel copies the batch's offset arrays (list offsets, and the query
+// offsets on the verification path) into the still unused ring: they must fit it.
+bool offsets_fit_ring(int64_t batch, bool verify, int ring_slots) {
+    return (batch + 1) * (verify ? 2 : 1) * (int64_t)sizeof(int32_t) <= (int64_t)ring_slots * kPageHeadBytes;
 }
 
 #define KAP_CUDA(call)                                                                         \
@@ -121,6 +173,9 @@ int g_trace_cap = 0, g_trace_next = 0;
 kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pages,
                             kap_workspace* ws, cudaStream_t stream) {
     if (ws->n_items == 0) return KAP_OK;
+    int cur_dev = -1;
+    if (cudaGetDevice(&cur_dev) != cudaSuccess || cur_dev != ws->device)
+        return fail(KAP_ERR_INVALID_ARG, "the workspace belongs to device %d but device %d is current", ws->device, cur_dev);
     const CUtensorMap* map = nullptr;
     kap_status st = get_tensor_map(ws, pool, pages, p_in.Hkv, &map);
     if (st != KAP_OK) return st;
@@ -145,7 +200,8 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     // the dependency wait) must not overlap the writer: one ordinary launch, then back to normal
     const bool use_pdl = g_use_pdl.load() && !ws->plain_next;
     ws->plain_next = 0;
-    p.early_kv = (use_pdl && g_early_kv.load() && !g_no_early_once.exchange(0)) ? 1 : 0;
+    const bool after_bulk_write = take_bulk_mark(ws, stream);
+    p.early_kv = (use_pdl && g_early_kv.load() && !after_bulk_write) ? 1 : 0;
 #ifdef KAP_TRACE
     p.trace = (g_trace && g_trace_next < g_trace_cap) ? g_trace + (size_t)(g_trace_next++) * 8192 * 8 : nullptr;
 #endif
@@ -229,7 +285,12 @@ extern "C" kap_status kap_workspace_create(kap_workspace** out, int32_t device, 
         max_rows_per_item > kRowTile * kMaxRowTiles)
         return fail(KAP_ERR_INVALID_ARG, "workspace sizes (%d items, %d rows, %d sequences)", max_items,
                     max_rows_per_item, max_batch);
-    KAP_CUDA(cudaSetDevice(device));
+    if (!offsets_fit_ring(max_batch, true, kDefaultSlots))
+        return fail(KAP_ERR_CAPACITY, "max_batch %d: a kernel stages the batch's offset arrays in %d bytes of shared "
+                    "memory, which holds %d sequences", max_batch, kDefaultSlots * kPageHeadBytes,
+                    kDefaultSlots * kPageHeadBytes / 8 - 1);
+    DeviceScope scope(device);                    // the caller's current device is put back on return
+    KAP_CUDA(scope.err);
     cudaDeviceProp prop;
     KAP_CUDA(cudaGetDeviceProperties(&prop, device));
     if (prop.major != 10)
@@ -296,8 +357,12 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     int32_t max_chunk = 0, row_tiles = 1;
     // resident CTAs per SM for the chosen ring size decide how many items make one wave;
     // clusters of 2, 4, 8 CTAs fit a few less (GPC boundaries)
-    KAP_CUDA(cudaSetDevice(ws->device));
+    DeviceScope scope(ws->device);                // the caller's current device is put back on return
+    KAP_CUDA(scope.err);
     const int ring_slots = g_ring_slots.load();
+    if (!offsets_fit_ring(batch, n_q != nullptr, ring_slots))
+        return fail(KAP_ERR_CAPACITY, "batch %d: the kernel stages the batch's offset arrays in its %d-slot ring "
+                    "(%d bytes)", batch, ring_slots, ring_slots * kPageHeadBytes);
     const int smem = smem_bytes_for(ring_slots);
     cudaFuncSetAttribute(kap_attn_split_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          smem_bytes_for(kMaxSlots));
@@ -306,10 +371,10 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         occ = 1;
     const int want = g_ctas_per_sm.load();
     const int per_sm = want > 0 ? std::min(want, occ) : occ;
-    ws->occupancy = occ;
-    ws->ring_slots = ring_slots;
-    ws->ctas_per_wave = per_sm * ws->sm_count;
-    int32_t slots[kMaxCluster] = {ws->ctas_per_wave};
+    // (nothing of the workspace changes until the new schedule is complete: a failure below leaves
+    // the previous schedule, ring size and cluster size in force together)
+    const int32_t ctas_per_wave = per_sm * ws->sm_count;
+    int32_t slots[kMaxCluster] = {ctas_per_wave};
     cudaFuncSetAttribute(kap_attn_split_kernel<0, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     cudaGetLastError();
     for (int c = 2; c <= kMaxCluster; ++c) {
@@ -324,7 +389,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         cc.attrs = ca; cc.numAttrs = 1;
         int n = 0;
         if (cudaOccupancyMaxActiveClusters(&n, kap_attn_split_kernel<0, false>, &cc) != cudaSuccess) { n = 0; cudaGetLastError(); }
-        slots[c - 1] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ws->ctas_per_wave / c);
+        slots[c - 1] = (int32_t)std::min<int64_t>((int64_t)n * per_sm / occ, ctas_per_wave / c);
     }
     // A one-wave schedule of the proposal path leaves a third of the SM's CTA slots to the next
     // kernel's early CTAs: those kernels last 10-30 us and what the early CTAs prefetch is a large
@@ -352,7 +417,6 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         if (groups[i].n_splits > 1) ws->h_merge[n_merge++] = groups[i];
     }
     if (!items.empty()) std::memcpy(ws->h_items, items.data(), sizeof(WorkItem) * items.size());
-    KAP_CUDA(cudaSetDevice(ws->device));
     if (!items.empty()) {
         KAP_CUDA(cudaMemcpyAsync(ws->d_items, ws->h_items, sizeof(WorkItem) * items.size(),
                                  cudaMemcpyHostToDevice, stream));
@@ -363,6 +427,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
                                      cudaMemcpyHostToDevice, stream));
     }
     KAP_CUDA(cudaEventRecord((cudaEvent_t)ws->upload_event, stream));
+    ws->occupancy = occ; ws->ring_slots = ring_slots; ws->ctas_per_wave = ctas_per_wave;
     ws->batch = batch; ws->n_items = (int32_t)items.size(); ws->n_groups = (int32_t)groups.size();
     ws->n_merge_groups = n_merge; ws->max_chunk = max_chunk; ws->row_tiles = row_tiles;
     ws->num_q_heads = num_q_heads; ws->num_kv_heads = num_kv_heads; ws->has_nq = n_q != nullptr;
@@ -521,9 +586,12 @@ StaticLayout static_layout(int64_t n_items, int64_t n_groups, int rows) {
 
 // Every (sequence, KV head) gets exactly `splits` work items of near-equal length (some may be
 // empty when the list is shorter than `splits`); item and partial slot (seq * Hkv + g) * splits + s.
+// A slice longer than `slice_cap` pages (what one CTA of the attention kernel can hold) is cut to
+// slice_cap and reported in *status (1 << KAP_ERR_CAPACITY): the pages beyond the cut are not
+// attended to, so the caller must treat the output as invalid.
 __global__ void kap_static_build_items_kernel(const int32_t* __restrict__ list_indptr, int batch,
-                                              int hkv, int splits, WorkItem* items,
-                                              MergeGroup* groups) {
+                                              int hkv, int splits, int slice_cap, WorkItem* items,
+                                              MergeGroup* groups, int32_t* status) {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= batch * hkv * splits) return;
     const int s = idx % splits, grp = idx / splits, g = grp % hkv, b = grp / hkv;
@@ -533,6 +601,10 @@ __global__ void kap_static_build_items_kernel(const int32_t* __restrict__ list_i
     it.seq = b; it.kv_head = g;
     it.page_begin = s * base + min(s, rem);
     it.page_end = it.page_begin + base + (s < rem ? 1 : 0);
+    if (it.page_end - it.page_begin > slice_cap) {
+        it.page_end = it.page_begin + slice_cap;
+        atomicOr(status, 1 << KAP_ERR_CAPACITY);
+    }
     it.group = grp; it.split = idx; it.n_splits = splits; it.n_q = 1;
     items[idx] = it;
     if (s == 0) {
@@ -560,6 +632,9 @@ extern "C" kap_status kap_selected_decode_attn_static(
         return fail(KAP_ERR_UNSUPPORTED, "head counts %d / %d", num_q_heads, num_kv_heads);
     if (batch < 0 || num_splits < 1) return fail(KAP_ERR_INVALID_ARG, "batch %d / num_splits %d", batch, num_splits);
     if (batch == 0) return KAP_OK;
+    if (!offsets_fit_ring(batch, false, kDefaultSlots))
+        return fail(KAP_ERR_CAPACITY, "batch %d: the kernel stages the batch's offsets in %d bytes of shared memory",
+                    batch, kDefaultSlots * kPageHeadBytes);
     if (!q || !kv_pool || !plan_indptr || !plan_phys_pages || !ctx_len || !out || num_pool_pages <= 0)
         return fail(KAP_ERR_INVALID_ARG, "NULL pointer or empty pool");
     if (reinterpret_cast<uintptr_t>(kv_pool) & 15) return fail(KAP_ERR_INVALID_ARG, "kv_pool is not 16-byte aligned");
@@ -584,6 +659,9 @@ extern "C" kap_status kap_selected_decode_attn_static(
             void* ptr = nullptr;
             KAP_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
             KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel<0, false>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          smem_bytes_for(kMaxSlots)));
+            KAP_CUDA(cudaFuncSetAttribute(kap_attn_split_kernel<2, false>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           smem_bytes_for(kMaxSlots)));
             g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
@@ -631,14 +709,21 @@ extern "C" kap_status kap_selected_decode_attn_static(
     // is written by this call's split kernel first
     KAP_CUDA(cudaMemsetAsync(base, 0, 256, stream));
     const int threads = 128;
+    // without logical indices the kernel keeps physical page ids only and a CTA holds 2.5 times
+    // as many of them
+    const bool plain = plan_logical_pages == nullptr;
     kap_static_build_items_kernel<<<(unsigned)((n_items + threads - 1) / threads), threads, 0, stream>>>(
-        plan_indptr, batch, num_kv_heads, num_splits, reinterpret_cast<WorkItem*>(base + lay.items_off),
-        reinterpret_cast<MergeGroup*>(base + lay.groups_off));
+        plan_indptr, batch, num_kv_heads, num_splits, plain ? kPlainIds : kMaxIds,
+        reinterpret_cast<WorkItem*>(base + lay.items_off),
+        reinterpret_cast<MergeGroup*>(base + lay.groups_off), reinterpret_cast<int32_t*>(base));
     KAP_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
-    // plain launches: the work list was written by the kernel just before, so the split kernel
+    // ordinary launches: the work list was written by the kernel just before, so the split kernel
     // must not start early
-    kap_attn_split_kernel<0, false><<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
+    if (plain)
+        kap_attn_split_kernel<2, false><<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
+    else
+        kap_attn_split_kernel<0, false><<<(unsigned)n_items, kThreads, smem_bytes_for(kDefaultSlots), stream>>>(map, p);
     KAP_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     if (num_splits > 1) {

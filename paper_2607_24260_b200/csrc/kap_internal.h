@@ -55,6 +55,7 @@ struct kap_workspace {
     int32_t plain_next = 0;        // the page lists were just rewritten on the device: launch the
                                    // next attention kernel as an ordinary (fully ordered) one
     int64_t total_rows = 0;        // sum over sequences of n_q
+    unsigned long long bulk_overflows_seen = 0;   // see kv_written_in_bulk() in kap_attn.cu
     // host (pinned) staging and device copies
     kap::WorkItem* h_items = nullptr;
     kap::WorkItem* d_items = nullptr;
@@ -62,8 +63,6 @@ struct kap_workspace {
     kap::MergeGroup* d_groups = nullptr;
     kap::MergeGroup* h_merge = nullptr;      // only the groups with n_splits > 1
     kap::MergeGroup* d_merge = nullptr;
-    int32_t* h_qrow0 = nullptr;              // [batch] first q row of each sequence
-    int32_t* d_qrow0 = nullptr;
     float* d_part_o = nullptr;               // [max_items][max_rows][128]
     float* d_part_ml = nullptr;              // [max_items][max_rows][2]   (m in log2 units, l)
     int32_t* d_status = nullptr;             // device status word

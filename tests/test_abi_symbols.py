@@ -76,3 +76,15 @@ int main(void) {
                     "-Wl,-rpath," + os.path.dirname(lib)], check=True)
     out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout
     assert out.strip().endswith("| 0:17 1:3 2:9 4:5 5:30 6:2 | 44 0"), out
+
+
+def test_workspace_refuses_a_batch_whose_offsets_do_not_fit_a_cta():
+    """Every CTA of the attention kernel stages the batch's offset arrays in shared memory, so the
+    library refuses batches beyond what fits - before it touches CUDA (this runs without a GPU) -
+    instead of letting a kernel write past its shared memory."""
+    import ctypes as C
+    from paper_2607_24260_b200 import kap
+    handle = C.c_void_p()
+    st = kap.lib().kap_workspace_create(C.byref(handle), 0, 64, 4, 8192)
+    assert st == kap.ERR_CAPACITY and not handle.value
+    assert b"max_batch 8192" in kap.lib().kap_last_error()

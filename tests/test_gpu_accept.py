@@ -22,7 +22,7 @@ def _run(logits_np, indptr, proposed, stride_pad=0):
     kap.top3_accept(logits, gu.i32(indptr), gu.i32(proposed), top3, acc, nxt, ctx_len=ctx)
     torch.cuda.synchronize()
     # the commit step: every rejected proposal leaves the context
-    k = np.diff(indptr) - 1
+    k = np.maximum(np.diff(indptr) - 1, 0)          # a window without rows commits nothing
     np.testing.assert_array_equal(ctx.cpu().numpy(), 1000 + 10 * np.arange(len(k)) - (k - acc.cpu().numpy()))
     return top3.cpu().numpy(), acc.cpu().numpy(), nxt.cpu().numpy()
 
@@ -48,6 +48,24 @@ def test_top3_accept_matches_oracle(V, pad):
     proposed[bad] = (ref_top3[bad, 0] + 1 + ref_top3[bad, 1]) % V
     ref = brute.top3_accept(x, indptr, proposed)
     got = _run(x, indptr, proposed, pad)
+    for g, r, name in zip(got, ref, ("top3", "accepted", "next_token")):
+        np.testing.assert_array_equal(g, r, err_msg=name)
+
+
+@pytest.mark.parametrize("V", [7, 32000])
+def test_top3_accept_empty_windows(V):
+    """Windows without any row - first, in the middle and last in the batch - accept nothing, carry
+    -1, leave ctx_len alone and do not look at a neighbour's rows."""
+    rng = synth.rng_for(V, "accept-empty")
+    rows_per_seq = [0, 5, 0, 1, 3, 0]
+    indptr = np.concatenate([[0], np.cumsum(rows_per_seq)]).astype(np.int32)
+    rows = int(indptr[-1])
+    x = rng.standard_normal((rows, V)).astype(np.float32)
+    ref_top3, _, _ = brute.top3_accept(x, indptr, np.zeros(rows, dtype=np.int32))
+    proposed = ref_top3[:, 1].astype(np.int32)               # every proposal is acceptable
+    ref = brute.top3_accept(x, indptr, proposed)
+    assert ref[1].tolist() == [0, 4, 0, 0, 2, 0] and ref[2][[0, 2, 5]].tolist() == [-1, -1, -1]
+    got = _run(x, indptr, proposed)
     for g, r, name in zip(got, ref, ("top3", "accepted", "next_token")):
         np.testing.assert_array_equal(g, r, err_msg=name)
 

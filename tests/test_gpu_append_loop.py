@@ -157,3 +157,65 @@ def test_bulk_append_then_decode_sees_every_new_token():
         assert_close(gu.dev_bf16_to_f64(d_out), ref, what="decode after a bulk append")
         np.testing.assert_array_equal(d_ctx.cpu().numpy(), final)
     ws.close()
+
+
+def test_bulk_append_mark_belongs_to_its_stream():
+    """Two streams in one process.  Stream A: a busy attention kernel, a several-token append, then
+    the attention call that must see every new token.  Between A's append and A's attention the
+    host issues an attention call on stream B (another workspace, another batch).  B's launch must
+    not use up the "loads wait for the append" mark that belongs to A: A's output still matches
+    the oracle, every repetition."""
+    w, end = _cycle_case(6, 7, (1500, 2040, 900))
+    B, Hq, Hkv, d = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim
+    rng = synth.rng_for(6, "two-streams")
+    n_new = np.array([6, 7, 4], dtype=np.int32)
+    indptr = np.concatenate([[0], np.cumsum(n_new)]).astype(np.int32)
+    q_bits, pool_bits = synth.host_qkv(w, 6, q_rows=B, q_std=4.0)
+    k_new = synth.normal_bf16((int(n_new.sum()), Hkv, d), 0.5, rng)
+    v_new = synth.normal_bf16((int(n_new.sum()), Hkv, d), 0.5, rng)
+    final = (w.ctx_len + n_new).astype(np.int32)
+    plan = kap.compile_plan(final, w.span_indptr, w.span_start, w.span_len, w.span_score,
+                            w.budget_tokens + 7, w.n_sink, w.n_recent + 7, None, 1.0, w.bt_indptr, w.bt_pages)
+    pool = gu.bits_to_dev(pool_bits)
+    d_ctx, d_q = gu.i32(w.ctx_len), gu.bits_to_dev(q_bits)
+    d_out = torch.zeros_like(d_q)
+    ws_a = kap.Workspace(max_rows_per_item=Hq // Hkv, max_batch=B)
+    ws_a.schedule(np.diff(plan["plan_indptr"]), None, Hq, Hkv)
+    args = (gu.i32(plan["plan_indptr"]), gu.i32(plan["plan_phys_pages"]), gu.i32(plan["plan_logical_pages"]))
+    d_k, d_v, d_ind = gu.bits_to_dev(k_new), gu.bits_to_dev(v_new), gu.i32(indptr)
+    d_bt_indptr, d_bt_pages = gu.i32(w.bt_indptr), gu.i32(w.bt_pages)
+    # stream B's own, unrelated work
+    wb = synth.config2(7, batch=2, L=3000, layers=1)
+    qb_bits, poolb_bits = synth.host_qkv(wb, 7, q_rows=2)
+    planb = kap.compile_workload(wb)
+    poolb, d_qb = gu.bits_to_dev(poolb_bits), gu.bits_to_dev(qb_bits)
+    d_outb = torch.zeros_like(d_qb)
+    ws_b = kap.Workspace(max_rows_per_item=Hq // Hkv, max_batch=2)
+    ws_b.schedule(np.diff(planb["plan_indptr"]), None, Hq, Hkv)
+    argsb = (gu.i32(planb["plan_indptr"]), gu.i32(planb["plan_phys_pages"]), gu.i32(planb["plan_logical_pages"]),
+             gu.i32(wb.ctx_len))
+    ref_b, _ = gu.oracle_decode(qb_bits, poolb_bits, planb, wb.ctx_len)
+    host_pool = pool_bits.copy()
+    for b in range(B):
+        bt = w.bt_pages[w.bt_indptr[b]:w.bt_indptr[b + 1]]
+        brute.append_kv(host_pool, bt, int(w.ctx_len[b]), k_new[indptr[b]:indptr[b + 1]], v_new[indptr[b]:indptr[b + 1]])
+    ref_a, _, _, _ = orc.selected_decode_attn(q_bits, host_pool, plan["plan_indptr"], plan["plan_phys_pages"],
+                                              plan["plan_logical_pages"], final)
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(4):                                      # repeat: a race would be intermittent
+        pool.copy_(gu.bits_to_dev(pool_bits))
+        d_ctx.copy_(gu.i32(w.ctx_len))
+        torch.cuda.synchronize()
+        kap.selected_decode_attn(d_q, pool, *args, d_ctx, d_out, ws_a, stream=sa)      # keeps A busy in front
+        kap.append_kv(d_k, d_v, pool, d_bt_indptr, d_bt_pages, d_ctx, new_indptr=d_ind, advance=True, stream=sa)
+        kap.selected_decode_attn(d_qb, poolb, *argsb, d_outb, ws_b, stream=sb)         # the intruder
+        kap.selected_decode_attn(d_q, pool, *args, d_ctx, d_out, ws_a, stream=sa)
+        torch.cuda.synchronize()
+        ws_a.check()
+        ws_b.check()
+        assert_close(gu.dev_bf16_to_f64(d_out), ref_a, what="stream A decode after its bulk append")
+        assert_close(gu.dev_bf16_to_f64(d_outb), ref_b, what="stream B decode")
+        np.testing.assert_array_equal(d_ctx.cpu().numpy(), final)
+    ws_a.close()
+    ws_b.close()
