@@ -153,3 +153,57 @@ def materialize_view(pool_bits, plan_phys_pages):
     page i holds the plan's i-th page; returns (compact pool, compact page ids)."""
     phys = np.asarray(plan_phys_pages, dtype=np.int64)
     return pool_bits[phys].copy(), np.arange(len(phys), dtype=np.int32)
+
+
+# reasons for falling back to full-context access (Section 3.2, "Runtime stability and fallback")
+FB_CAPACITY, FB_METADATA, FB_CONFIDENCE, FB_S_HIGH, FB_H_LOW, FB_NO_MARGIN, FB_SLACK = 1, 2, 4, 8, 16, 32, 64
+RT_OVER_CAPACITY, RT_UNSTABLE_METADATA = 1, 2     # runtime_flags given by the caller
+_PLAN_S_HIGH = 4                                  # the compiler's "retained ratio above s_max" flag
+
+
+def fallback_decide(accepted_sum, proposed_sum, min_proposed, h_prior, s, kv, w_main, w_prop,
+                    h_min, s_max, plan_flags=None, runtime_flags=None, confidence=None,
+                    confidence_min=0.0):
+    """The fallback rule of Section 3.2 ("Runtime stability and fallback") with the quantities of
+    Section 4, one sequence at a time.  A sequence takes full-context access when
+      * its plan exceeds the compact workspace, or breaks the metadata-stability assumptions
+        (both reported by the caller in runtime_flags),
+      * its prior confidence is below confidence_min,
+      * it retains too much KV: s > s_max, or the compiler already flagged that,
+      * its observed acceptance is low: h < h_min, where h = accepted / proposed (Eq. 5) once at
+        least min_proposed proposals were verified and h_prior before that,
+      * h <= s: no KV-side margin (Eq. 11), whatever the context length,
+      * the phase slack of Eq. 13, h (W_main + KV) - (W_prop + s KV), is not positive.
+    Besides the decision the function returns the slack and the factor by which s could be
+    multiplied before the slack reaches zero (room to widen the budget when > 1, the cut needed when
+    < 1): scale = (h (W_main + KV) - W_prop) / (s KV).
+    Returns a list of dicts: force_full, reasons, h, slack, budget_scale."""
+    res = []
+    for b in range(len(s)):
+        n_prop, n_acc = int(proposed_sum[b]), int(accepted_sum[b])
+        h = n_acc / n_prop if n_prop >= max(int(min_proposed), 1) else float(h_prior)
+        kv_b, s_b = float(kv[b]), float(s[b])
+        slack = h * (w_main + kv_b) - (w_prop + s_b * kv_b)
+        room = h * (w_main + kv_b) - w_prop
+        if s_b * kv_b > 0:
+            scale = max(room, 0.0) / (s_b * kv_b)
+        else:
+            scale = float("inf") if room > 0 else 0.0
+        why = 0
+        rt = 0 if runtime_flags is None else int(runtime_flags[b])
+        if rt & RT_OVER_CAPACITY:
+            why |= FB_CAPACITY
+        if rt & RT_UNSTABLE_METADATA:
+            why |= FB_METADATA
+        if confidence is not None and float(confidence[b]) < confidence_min:
+            why |= FB_CONFIDENCE
+        if s_b > s_max or (plan_flags is not None and int(plan_flags[b]) & _PLAN_S_HIGH):
+            why |= FB_S_HIGH
+        if h < h_min:
+            why |= FB_H_LOW
+        if h <= s_b:
+            why |= FB_NO_MARGIN
+        if not slack > 0:
+            why |= FB_SLACK
+        res.append(dict(force_full=1 if why else 0, reasons=why, h=h, slack=slack, budget_scale=scale))
+    return res
