@@ -347,6 +347,65 @@ kap_status kap_top3_accept(
 kap_status kap_phase_model(double k, double h, double s, double w_main, double w_prop, double kv,
                            double* out /* HOST [8] */);
 
+/* runtime conditions the caller reports to kap_fallback_decide (bit-or) */
+enum {
+    KAP_RUNTIME_OVER_CAPACITY = 1,     /* the plan did not fit the space reserved for it (a compile
+                                          or view call returned KAP_ERR_CAPACITY) */
+    KAP_RUNTIME_UNSTABLE_METADATA = 2  /* list lengths / shapes changed so that the captured graphs
+                                          and the schedule no longer apply */
+};
+/* why kap_fallback_decide sends a sequence to full-context access (bit-or) */
+enum {
+    KAP_FALLBACK_CAPACITY = 1, KAP_FALLBACK_METADATA = 2, KAP_FALLBACK_CONFIDENCE = 4,
+    KAP_FALLBACK_S_HIGH = 8, KAP_FALLBACK_H_LOW = 16, KAP_FALLBACK_NO_MARGIN = 32,
+    KAP_FALLBACK_SLACK = 64
+};
+
+/*
+ * kap_fallback_decide - the fallback rule of Section 3.2 ("Runtime stability and fallback") with
+ * the quantities of Section 4: the executor returns a request to full-context access when its plan
+ * exceeds the compact workspace, breaks the metadata-stability assumptions, comes from priors of
+ * too little confidence, retains too much KV (s high) or is accepted too rarely (h low); Section 4.2
+ * adds that observed acceptance and profiled costs decide when the phase slack has turned
+ * unfavourable.  HOST only, per sequence b:
+ *   h      = accepted_sum[b] / proposed_sum[b] (Eq. 5; the running sums of kap_top3_accept's
+ *            accepted[] and of the proposals verified) once proposed_sum[b] >= max(min_proposed, 1),
+ *            h_prior before that
+ *   slack  = h (w_main + kv[b]) - (w_prop + s[b] kv[b])                              (Eq. 13)
+ *   reasons (bit-or): CAPACITY / METADATA from runtime_flags[b]; CONFIDENCE when confidence[b] <
+ *            confidence_min; S_HIGH when s[b] > s_max or plan_flags[b] has KAP_PLAN_S_HIGH;
+ *            H_LOW when h < h_min; NO_MARGIN when h <= s[b] (Eq. 11: no context length can make
+ *            such a plan pay); SLACK when slack <= 0 (Eq. 8).
+ *   force_full[b] = 1 iff any reason applies - feed it to kap_compile_plan's force_full for the
+ *            next cycle (the identity plan through the same kernels).
+ *   budget_scale[b] = (h (w_main + kv) - w_prop) / (s kv), floored at 0: the factor by which s
+ *            could be multiplied before the slack reaches zero - room to widen the budget when
+ *            > 1, the cut that would bring the plan back to break-even when < 1 (the paper's
+ *            "budget adjustment"; +inf when s kv = 0 and there is room).
+ * Costs are in any one unit: bytes, or measured times (attention only: w_main = w_prop = 0,
+ * kv[b] = the sequence's share of the measured full-context decode time, s[b] = measured
+ * proposal time / full time, or the page ratio kap_compile_plan realised).
+ * plan_flags, runtime_flags, confidence, reasons, h_used, slack and budget_scale may be NULL.
+ * Errors: KAP_ERR_INVALID_ARG (NULL pointer, negative batch, NaN, h_prior outside [0, 1],
+ * negative or non-finite costs, more accepted than proposed); outputs untouched on error.
+ */
+kap_status kap_fallback_decide(
+    int32_t batch,
+    const int64_t* accepted_sum,       /* HOST [batch] */
+    const int64_t* proposed_sum,       /* HOST [batch] */
+    int64_t min_proposed, double h_prior,
+    const double* s,                   /* HOST [batch] retained-KV ratio (Eq. 4) */
+    const double* kv,                  /* HOST [batch] cost of reading the sequence's whole KV */
+    double w_main, double w_prop,
+    double h_min, double s_max,
+    const int32_t* plan_flags,         /* HOST [batch] KAP_PLAN_* or NULL */
+    const int32_t* runtime_flags,      /* HOST [batch] KAP_RUNTIME_* or NULL */
+    const double* confidence,          /* HOST [batch] or NULL */
+    double confidence_min,
+    uint8_t* force_full,               /* HOST out [batch] */
+    int32_t* reasons,                  /* HOST out [batch] or NULL */
+    double* h_used, double* slack, double* budget_scale);   /* HOST out [batch] or NULL */
+
 /*
  * kap_compile_growing_plan / kap_refresh_recent - one compiled plan for a context that grows
  * (Section 3.2: k proposal steps per cycle, many cycles per request; the plan is compiled once per

@@ -52,6 +52,12 @@ SIGNATURES = {
     "kap_top3_accept": (C.c_int, [_vp, C.c_int64, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
                                   _vp, _vp, _vp]),
     "kap_phase_model": (C.c_int, [C.c_double] * 6 + [C.POINTER(C.c_double)]),
+    "kap_fallback_decide": (C.c_int, [C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.c_int64,
+                                      C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                      C.c_double, C.c_double, C.c_double, C.c_double, _i32p, _i32p,
+                                      C.POINTER(C.c_double), C.c_double, _u8p, _i32p,
+                                      C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                      C.POINTER(C.c_double)]),
     "kap_materialize_view": (C.c_int, [_vp, C.c_int64, _vp, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                        _vp, C.c_int64, _vp, _vp, _vp]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
@@ -359,6 +365,31 @@ def phase_model(k, h, s, w_main, w_prop, kv):
     out = (C.c_double * 8)()
     _check(lib().kap_phase_model(float(k), float(h), float(s), float(w_main), float(w_prop), float(kv), out))
     return dict(zip(PHASE_FIELDS, [float(x) for x in out]))
+
+
+FALLBACK_CAPACITY, FALLBACK_METADATA, FALLBACK_CONFIDENCE, FALLBACK_S_HIGH, FALLBACK_H_LOW, \
+    FALLBACK_NO_MARGIN, FALLBACK_SLACK = 1, 2, 4, 8, 16, 32, 64
+RUNTIME_OVER_CAPACITY, RUNTIME_UNSTABLE_METADATA = 1, 2
+
+
+def fallback_decide(accepted_sum, proposed_sum, s, kv, w_main=0.0, w_prop=0.0, min_proposed=1,
+                    h_prior=1.0, h_min=0.0, s_max=1.0, plan_flags=None, runtime_flags=None,
+                    confidence=None, confidence_min=0.0):
+    """kap_fallback_decide on host arrays; returns a dict of numpy arrays: force_full (uint8, ready
+    for compile_plan's force_full), reasons, h, slack, budget_scale."""
+    acc, prop = _np(accepted_sum, np.int64), _np(proposed_sum, np.int64)
+    s, kv = _np(s, np.float64), _np(kv, np.float64)
+    B = int(s.shape[0])
+    flags, rt, conf = _np(plan_flags, np.int32), _np(runtime_flags, np.int32), _np(confidence, np.float64)
+    out = dict(force_full=np.zeros(B, dtype=np.uint8), reasons=np.zeros(B, dtype=np.int32),
+               h=np.zeros(B), slack=np.zeros(B), budget_scale=np.zeros(B))
+    _check(lib().kap_fallback_decide(
+        B, _ptr(acc, C.c_int64), _ptr(prop, C.c_int64), int(min_proposed), float(h_prior),
+        _ptr(s, C.c_double), _ptr(kv, C.c_double), float(w_main), float(w_prop), float(h_min),
+        float(s_max), _ptr(flags, C.c_int32), _ptr(rt, C.c_int32), _ptr(conf, C.c_double),
+        float(confidence_min), _ptr(out["force_full"], C.c_uint8), _ptr(out["reasons"], C.c_int32),
+        _ptr(out["h"], C.c_double), _ptr(out["slack"], C.c_double), _ptr(out["budget_scale"], C.c_double)))
+    return out
 
 
 def materialize_view(kv_pool, plan_phys_pages, compact_pool, compact_pages=None, device_status=None,
