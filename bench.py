@@ -12,11 +12,17 @@ compilation and scheduling on the host, host->device copies of plan arrays and q
 device->host copy of every attention output, all inside the timed region (the KV cache itself is
 persistent state and stays on the device).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--no-sweep]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c4] [--no-sweep]
     python bench.py --impl reference ...      # the CPU oracle on the same metric (rank 0 only)
+    python bench.py --impl host-plan ...      # host leg only (plan compilation), runs without a GPU
 
-N > 1: one process per GPU (torchrun), every rank runs its own batch (weak scaling, no data-path
-collective); time = max over ranks.
+The headline workload is configuration 4 (B = 4, 128K context, all 32 layers, 68.7 GB of KV: the
+largest single-GPU configuration, inside the 32K-128K range the target is stated on);
+configuration 3 is measured beside it in full, configurations 2, 5 and 1 as side lines.
+
+N > 1: one process per GPU, every rank runs its own batch (weak scaling, no data-path
+collective); time = max over ranks.  Under torchrun the ranks come from the environment; a plain
+`python bench.py --gpus N` starts its own N ranks through torch.distributed.run.
 """
 from __future__ import annotations
 
@@ -38,10 +44,13 @@ if ROOT not in sys.path:
 METRIC = "plan-guided decode attn tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read+write per launch / algorithmic bytes per launch, from the ncu captures
-# summarised under profiles/kap_attn_split_kernel_c2_c3_c4.md (c2 captured with 4 of its 32 layers;
-# traffic per launch does not depend on the layer count)
-TRAFFIC_RATIO = {"decode": 1.018, "verify": 1.007}
+
+
+def traffic_ratios():
+    """dram__bytes_read+write per launch / algorithmic bytes per launch from the last ncu capture
+    (profiles/traffic_ratio.txt); None when that capture was taken on other kernel sources"""
+    from paper_2607_24260_b200 import traffic
+    return traffic.read_ratios()
 
 
 def measured_peak():
@@ -215,25 +224,48 @@ class Cycle:
         self.ws_d.check()
         self.ws_v.check()
 
-    def time_steps(self, steps, warmup):
-        """Returns (total_ms, decode_segment_ms, verify_segment_ms) over `steps` cycles."""
+    def time_steps(self, steps, warmup, min_replays=20, min_seconds=0.5):
+        """Times EXACTLY `steps` cycles (total and per segment), then goes on replaying until at
+        least `min_replays` cycles and `min_seconds` of device time have been timed, for the
+        per-step statistics.  Returns (total_ms, decode_ms, verify_ms) of the first `steps` cycles
+        and a dict with mean / median / best over all timed cycles."""
         torch = self.torch
         for _ in range(warmup):
             self.graph_d.replay()
             self.graph_v.replay()
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
-        torch.cuda.synchronize()
-        for s in range(steps):
-            ev[s][0].record()
-            self.graph_d.replay()
-            ev[s][1].record()
-            self.graph_v.replay()
-            ev[s][2].record()
-        torch.cuda.synchronize()
-        total = ev[0][0].elapsed_time(ev[-1][2])
-        dec = sum(e[0].elapsed_time(e[1]) for e in ev)
-        ver = sum(e[1].elapsed_time(e[2]) for e in ev)
-        return total, dec, ver
+
+        def timed(n):
+            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n)]
+            torch.cuda.synchronize()
+            for s in range(n):
+                ev[s][0].record()
+                self.graph_d.replay()
+                ev[s][1].record()
+                self.graph_v.replay()
+                ev[s][2].record()
+            torch.cuda.synchronize()
+            dec = [e[0].elapsed_time(e[1]) for e in ev]
+            ver = [e[1].elapsed_time(e[2]) for e in ev]
+            return ev[0][0].elapsed_time(ev[-1][2]), dec, ver
+
+        total, dec, ver = timed(steps)
+        all_dec, all_ver = list(dec), list(ver)
+        per_step = total / steps
+        more = max(min_replays - steps, int(min_seconds * 1e3 / max(per_step, 1e-6)) + 1 - steps, 0)
+        if more:
+            _, d2, v2 = timed(more)
+            all_dec += d2
+            all_ver += v2
+        cyc = [d + v for d, v in zip(all_dec, all_ver)]
+        us_d = lambda ms: ms / (self.k * self.layers) * 1e3
+        us_v = lambda ms: ms / self.layers * 1e3
+        stats = {"replays": len(cyc), "timed_seconds": round(sum(cyc) * 1e-3, 3),
+                 "cycle_ms": {"mean": statistics.fmean(cyc), "median": statistics.median(cyc), "best": min(cyc)},
+                 "us_per_layer_decode": {"mean": us_d(statistics.fmean(all_dec)), "median": us_d(statistics.median(all_dec)),
+                                         "best": us_d(min(all_dec))},
+                 "us_per_layer_verify": {"mean": us_v(statistics.fmean(all_ver)), "median": us_v(statistics.median(all_ver)),
+                                         "best": us_v(min(all_ver))}}
+        return total, sum(dec), sum(ver), stats
 
     def free(self):
         for ws in (self.ws_d, self.ws_v):
@@ -252,8 +284,10 @@ def summarise(cy: Cycle, steps, total_ms, dec_ms, ver_ms, n_ranks=1):
     gbs_dec = cy.decode_bytes / (us_dec_layer * 1e-6) / 1e9
     gbs_ver = cy.verify_bytes / (us_ver_layer * 1e-6) / 1e9
 
+    ratios = traffic_ratios()
+
     def roof(kind, gbs, alg_bytes):
-        ratio = TRAFFIC_RATIO[kind]
+        ratio = ratios[kind]
         return {"bound": "hbm", "kernel": f"kap_attn_split_kernel ({kind} launch incl. its merge pass)",
                 "achieved": round(gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(gbs / peak, 4),
                 "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4), "peak_kind": f"of {peak_kind}",
@@ -530,11 +564,11 @@ class OracleSampler:
         return float(self.w.layers * (k * dec.sum() + ver.sum()))
 
 
-def cpu_baseline(w, k, budget_s=12.0):
+def cpu_baseline(w, k, budget_s=12.0, min_units=None):
     sm = OracleSampler(w)
-    spent = sm.run_units(w.batch)                       # every sequence once
+    spent = sm.run_units(w.batch if min_units is None else min_units)   # by default every sequence once
     while spent < budget_s and sm.units < w.batch * w.layers:
-        spent += sm.run_units(w.batch)
+        spent += sm.run_units(1 if min_units is not None else w.batch)
     cycle_s = sm.cycle_seconds(k)
     return {"value": w.batch * k / cycle_s, "unit": "tokens/s", "cores": sm.threads, "kind": "oracle",
             "sample": f"{sm.units} (sequence, layer) units of {w.name}'s {w.batch * w.layers} (each: proposal-pass "
@@ -566,6 +600,30 @@ def config_dict(w, k, layers, extra=None):
     return c
 
 
+def oracle_sample_main(args):
+    """--oracle-sample S: time the oracle for about S seconds on the named configuration and print
+    the cpu_baseline dict (used by the parent to get a single-thread figure: the child runs with
+    OMP_NUM_THREADS=1)."""
+    from paper_2607_24260_b200 import synth
+    w = synth.CONFIGS[args.config](0)
+    print(json.dumps(cpu_baseline(w, int(w.n_q.max()), budget_s=args.oracle_sample, min_units=1)))
+    return 0
+
+
+def cpu_baseline_single_thread(config, budget_s=6.0):
+    """the same oracle, one thread: a child process with OMP_NUM_THREADS=1"""
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    for key in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+        env.pop(key, None)
+    try:
+        out = subprocess.run([sys.executable, os.path.abspath(__file__), "--config", config,
+                              "--oracle-sample", str(budget_s)], env=env, capture_output=True, text=True,
+                             timeout=600, check=True).stdout
+        return json.loads(out.strip().splitlines()[-1])
+    except Exception as e:
+        return {"error": repr(e)}
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle on the same metric and workload (rank 0 only; the other
     ranks exit without work).  Each step times a bounded sample of (sequence, layer) units, sized
@@ -589,7 +647,7 @@ def run_reference(args):
     sample = (f"{units_per_step} (sequence, layer) units per step, {sm.units} sampled in total (the workload has {w.batch * w.layers}; repeats allowed), "
               f"scaled to the full cycle")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s",
-            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+            "n_gpus": max(world, args.gpus), "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": config_dict(w, k, w.layers),
             "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": sm.threads, "kind": "oracle",
@@ -600,17 +658,169 @@ def run_reference(args):
     return 0
 
 
+def run_host_plan(args):
+    """--impl host-plan: the host leg of the path only - kap_compile_plan on every rank's own batch
+    (no GPU work, so it runs anywhere; backend gloo without CUDA).  It exists so that the launch,
+    sharding, barrier and max-over-ranks plumbing the GPU arm uses can be run on a CPU machine."""
+    import torch
+    from paper_2607_24260_b200 import dist as kdist, kap, synth
+    rank, local_rank, world = dist_env()
+    group = None
+    if world > 1:
+        cuda = torch.cuda.is_available()
+        group = kdist.Group("nccl" if cuda else "gloo", device=f"cuda:{local_rank}" if cuda else "cpu")
+    base = synth.CONFIGS[args.config](0, layers=1) if args.config != "c1" else synth.CONFIGS["c1"](0)
+    lo, hi = kdist.shard_units(world * base.batch, rank, world)     # this rank's sequences of the global batch
+    w = synth.CONFIGS[args.config](lo // base.batch, layers=1) if args.config != "c1" else base
+    for _ in range(max(3, args.warmup)):
+        kap.compile_workload(w)
+    if group:
+        group.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        plan = kap.compile_workload(w)
+    elapsed = time.perf_counter() - t0
+    units = float((hi - lo) * args.steps)
+    if group:
+        group.barrier()
+        value = kdist.aggregate_throughput(units, elapsed, group)
+        slowest = group.max_float(elapsed)
+    else:
+        value, slowest = units / elapsed, elapsed
+    if rank == 0:
+        print(json.dumps({"impl": "host-plan", "metric": "plans compiled per second (host leg only)", "value": value,
+                          "unit": "sequences/s", "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+                          "ms_per_step": slowest / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+                          "config": {"workload": f"{w.name}: {w.note}", "sequences_per_rank": hi - lo,
+                                     "pages_selected_rank0": int(plan["plan_indptr"][-1])}}))
+    if group:
+        group.close()
+    return 0
+
+
+def self_launch(args):
+    """`python bench.py --gpus N` without torchrun: start the N ranks ourselves"""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def measure(name, args, dev, seed, group, world, layers=None, want_e2e=True, want_extras=False):
+    """One configuration: device-resident cycle timing (exactly args.steps cycles, then the
+    per-step statistics), optionally e2e and the side calls.  Returns (result dict, Cycle)."""
+    import torch
+    cy = Cycle(name, seed=seed, layers=layers, device=dev, kv_layout=args.kv_layout,
+               decode_chunk=args.decode_chunk, verify_chunk=args.verify_chunk)
+    cy.capture()
+    if group:
+        group.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(int(dev.split(":")[1])) as clocks:
+        total_ms, dec_ms, ver_ms, stats = cy.time_steps(args.steps, max(3, args.warmup))
+    torch.cuda.synchronize()
+    local_ms = total_ms
+    if group:
+        from paper_2607_24260_b200 import dist as kdist
+        group.barrier()
+        total_ms = group.max_float(total_ms)
+    res = summarise(cy, args.steps, total_ms, dec_ms, ver_ms, n_ranks=world)
+    if group:      # all ranks' tokens / the slowest rank's time, through the tested helper
+        res["tokens_per_s"] = kdist.aggregate_throughput(float(cy.w.batch * cy.k * args.steps), local_ms * 1e-3, group)
+    res["per_step"] = stats
+    res["clocks"] = clocks.summary()
+    if want_e2e:
+        e2e_ms, h2d, d2h = time_e2e(cy, max(3, min(args.steps, 20)), 3)
+        if group:
+            e2e_ms = group.max_float(e2e_ms)
+        res["e2e"] = {"value": world * cy.w.batch * cy.k / (e2e_ms * 1e-3), "unit": "tokens/s",
+                      "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                      "note": "per step: host plan compile (Algorithm 1) + both kap_schedule calls (list lengths "
+                              "unchanged, so they return without rebuilding: a schedule is per request shape, "
+                              "its uncached cost is other_calls.schedule_ms) + H2D of plan arrays, ctx_len and "
+                              "every query + the cycle + D2H of every attention output; the KV cache is "
+                              "device-resident state"}
+    cy.ws_d.check()
+    cy.ws_v.check()
+    res["gpu_launches"] = cy.launches_per_step * stats["replays"]
+    if want_extras:
+        res["other_calls"] = time_extras(cy)
+        from paper_2607_24260_b200 import kap
+        res["phase"] = phase_report(kap, cy.k, res["us_per_layer_decode"], res["us_per_layer_verify"],
+                                    res["other_calls"]["full_decode_us_per_layer"])
+    return res, cy
+
+
+def side_entry(r, cy):
+    out = {"workload": cy.w.note, "layers_timed": cy.layers, "replays": r["per_step"]["replays"],
+           "timed_seconds": r["per_step"]["timed_seconds"],
+           "us_per_layer_decode": r["us_per_layer_decode"], "us_per_layer_verify": r["us_per_layer_verify"],
+           "us_per_layer_decode_median_best": [round(r["per_step"]["us_per_layer_decode"][x], 3) for x in ("median", "best")],
+           "us_per_layer_verify_median_best": [round(r["per_step"]["us_per_layer_verify"][x], 3) for x in ("median", "best")],
+           "decode_GBps": r["decode"]["achieved"], "verify_GBps": r["verify"]["achieved"],
+           "decode_frac_of_measured": r["decode"]["frac"], "decode_frac_of_8TBs": r["decode"]["frac_of_nominal_8TBs"],
+           "verify_frac_of_measured": r["verify"]["frac"], "verify_frac_of_8TBs": r["verify"]["frac_of_nominal_8TBs"],
+           "retained_kv_ratio_s": r["retained_kv_ratio_s"], "decode_only_tokens_per_s": r["decode_only_tokens_per_s"],
+           "tokens_per_s": r["tokens_per_s"], "schedule": r["schedule"], "clocks": r["clocks"]}
+    for key in ("e2e", "cpu_baseline", "cpu_baseline_single_thread", "roofline_decode", "roofline_verify"):
+        if key in r:
+            out[key] = r[key]
+    return out
+
+
+def time_c1_warm_cold(args, dev):
+    """Configuration 1 (one sequence, one layer, 4096 tokens): its 16.8 MB of KV stay in the L2
+    between replays, so one proposal pass and the verification pass are timed twice - replayed
+    back to back (warm) and with a 512 MB buffer streamed before every replay (cold: the KV comes
+    from HBM again).  Launch-latency bound either way."""
+    import torch
+    cy = Cycle("c1", seed=0, device=dev, kv_layout=args.kv_layout)
+    cy.capture()
+    g1 = torch.cuda.CUDAGraph()                       # ONE proposal pass (the cycle's graph holds k)
+    stream = torch.cuda.Stream(device=dev)
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g1, stream=stream):
+        cy.kap.selected_decode_attn(cy.q_dec[0, 0], cy.pool_attn[0], cy.d_plan_indptr, cy.d_plan_phys,
+                                    cy.d_plan_logical, cy.d_ctx, cy.out_dec[0, 0], cy.ws_d)
+    flush = torch.zeros(512 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(graph, cold):
+        t = []
+        for i in range(3 + 20):
+            if cold:
+                flush.add_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); graph.replay(); e1.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                t.append(e0.elapsed_time(e1) * 1e3)
+        return [round(statistics.median(t), 2), round(min(t), 2)]
+
+    out = {"workload": cy.w.note, "decode_bytes": cy.decode_bytes, "verify_bytes": cy.verify_bytes,
+           "note": "one layer, 16.8 MB of KV; [median, best] microseconds over 20 replays; warm = L2-resident, "
+                   "cold = 512 MB streamed before every replay; launch-latency bound, not a bandwidth figure"}
+    for mode in ("warm", "cold"):
+        out[mode] = {"decode_us": timed(g1, mode == "cold"), "verify_us": timed(cy.graph_v, mode == "cold")}
+    del flush
+    cy.free()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "host-plan"])
+    ap.add_argument("--config", default="c4", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (debugging)")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the 32K / 128K side measurements")
-    ap.add_argument("--sweep-layers", type=int, default=8)
-    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the other configurations")
+    ap.add_argument("--sweep-layers", type=int, default=None, help="layer count of the side configurations")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline legs")
+    ap.add_argument("--oracle-sample", type=float, default=0.0, help=argparse.SUPPRESS)
     ap.add_argument("--max-cluster", type=int, default=-1)
     ap.add_argument("--ring-slots", type=int, default=-1)
     ap.add_argument("--decode-chunk", type=int, default=0, help="cap on pages per CTA, proposal path")
@@ -621,8 +831,14 @@ def main():
     ap.add_argument("--kv-layout", default="hnd", choices=["hnd", "nhd"],
                     help="pool layout given to the attention calls (default: head-major)")
     args = ap.parse_args()
+    if args.oracle_sample > 0:
+        return oracle_sample_main(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        return self_launch(args)
     if args.impl == "reference":
         return run_reference(args)
+    if args.impl == "host-plan":
+        return run_host_plan(args)
 
     import torch
     from paper_2607_24260_b200 import kap
@@ -631,91 +847,71 @@ def main():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    dist = None
+    group = None
     if world > 1:
         from paper_2607_24260_b200 import dist as kdist
-        dist = kdist.Group("nccl", device=dev)
+        group = kdist.Group("nccl", device=dev)
+        lo, _ = kdist.shard_units(world * 1, rank, world)    # one batch per rank: weak scaling
+        seed = lo
+    else:
+        seed = 0
     kap.set_launch_options(args.pdl, args.early_kv, args.ctas_per_sm, args.max_cluster, args.ring_slots)
-    warmup = max(3, args.warmup)
+    solo = rank == 0 and world == 1
 
-    cy = Cycle(args.config, seed=rank, layers=args.layers, device=dev, kv_layout=args.kv_layout, decode_chunk=args.decode_chunk,
-               verify_chunk=args.verify_chunk)
-    cy.capture()
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    with ClockSampler(local_rank) as clocks:
-        total_ms, dec_ms, ver_ms = cy.time_steps(args.steps, warmup)
-    torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
-        total_ms = dist.max_float(total_ms)
-    res = summarise(cy, args.steps, total_ms, dec_ms, ver_ms, n_ranks=world)
-    e2e_ms, h2d, d2h = time_e2e(cy, max(3, min(args.steps, 20)), 3)
-    if dist:
-        e2e_ms = dist.max_float(e2e_ms)
-    cy.ws_d.check()
-    cy.ws_v.check()
-    extras = time_extras(cy) if (rank == 0 and world == 1) else None
+    res, cy = measure(args.config, args, dev, seed, group, world, layers=args.layers, want_extras=solo)
     w, k = cy.w, cy.k
     dominant = "verify" if res["share_decode"] < 0.5 else "decode"
     line = {
         "metric": METRIC, "value": res["tokens_per_s"], "unit": "tokens/s", "n_gpus": world,
-        "steps": args.steps, "warmup": warmup, "ms_per_step": res["ms_per_step"],
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": res["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": config_dict(w, k, cy.layers, {"parallelism": f"dp{world} (independent batches per GPU)",
                                                  "pdl": args.pdl, "max_cluster": args.max_cluster, "ring_slots": args.ring_slots,
                                                  "ctas_per_sm": args.ctas_per_sm, "early_kv": args.early_kv,
                                                  "kv_layout": args.kv_layout}),
-        "clocks": clocks.summary(),
-        "e2e": {"value": world * w.batch * k / (e2e_ms * 1e-3), "unit": "tokens/s",
-                "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "note": "host plan compile + schedule + H2D of plans/queries + cycle + D2H of outputs; "
-                        "the KV cache is device-resident state"},
-        "gpu_launches": cy.launches_per_step * args.steps,
+        "clocks": res["clocks"], "per_step": res["per_step"], "e2e": res["e2e"],
+        "gpu_launches": res["gpu_launches"],
         "roofline": res[dominant], "roofline_decode": res["decode"], "roofline_verify": res["verify"],
         "us_per_layer_decode": res["us_per_layer_decode"],
         "us_per_layer_verify": res["us_per_layer_verify"],
         "decode_only_tokens_per_s": res["decode_only_tokens_per_s"],
         "retained_kv_ratio_s": res["retained_kv_ratio_s"], "schedule": res["schedule"],
     }
-    if extras:
-        line["other_calls"] = extras
-        line["phase"] = phase_report(kap, cy.k, res["us_per_layer_decode"], res["us_per_layer_verify"],
-                                     extras["full_decode_us_per_layer"])
+    for key in ("other_calls", "phase"):
+        if key in res:
+            line[key] = res[key]
     cy.free()
 
-    if rank == 0 and world == 1 and not args.no_sweep and args.config == "c2":
-        sweep = {}
-        for name in ("c3", "c4", "c5"):
+    if solo and not args.no_sweep:
+        also = {}
+        plan = [n for n in ("c4", "c3", "c2", "c5") if n != args.config]
+        for name in plan:
             try:
-                c2 = Cycle(name, seed=0, layers=args.sweep_layers if name != "c5" else max(1, args.sweep_layers // 2),
-                           device=dev)
-                c2.capture()
-                n_side = max(5, min(40, args.steps // 4))
-                t, d, v = c2.time_steps(n_side, 3)
-                r = summarise(c2, n_side, t, d, v)
-                sweep[name] = {"workload": c2.w.note, "layers_timed": c2.layers,
-                               "us_per_layer_decode": r["us_per_layer_decode"],
-                               "us_per_layer_verify": r["us_per_layer_verify"],
-                               "decode_GBps": r["decode"]["achieved"], "verify_GBps": r["verify"]["achieved"],
-                               "decode_frac_of_measured": r["decode"]["frac"],
-                               "decode_frac_of_8TBs": r["decode"]["frac_of_nominal_8TBs"],
-                               "verify_frac_of_measured": r["verify"]["frac"],
-                               "verify_frac_of_8TBs": r["verify"]["frac_of_nominal_8TBs"],
-                               "retained_kv_ratio_s": r["retained_kv_ratio_s"],
-                               "decode_only_tokens_per_s": r["decode_only_tokens_per_s"]}
+                full = name in ("c3", "c4")                  # measured like the headline: e2e and CPU baseline too
+                layers = args.sweep_layers if args.sweep_layers else (None if name != "c5" else 4)
+                r, c2 = measure(name, args, dev, 0, None, 1, layers=layers, want_e2e=full)
+                if full and not args.no_cpu:
+                    r["cpu_baseline"] = cpu_baseline(c2.w, c2.k)
+                    r["cpu_baseline_single_thread"] = cpu_baseline_single_thread(name)
+                if full:
+                    r["roofline_decode"], r["roofline_verify"] = r["decode"], r["verify"]
+                also[name] = side_entry(r, c2)
                 c2.free()
             except Exception as e:       # a side measurement must not lose the main line
-                sweep[name] = {"error": repr(e)}
-        line["sweep"] = sweep
-    if rank == 0 and world == 1 and not args.no_cpu:
+                also[name] = {"error": repr(e)}
+        try:
+            also["c1"] = time_c1_warm_cold(args, dev)
+        except Exception as e:
+            also["c1"] = {"error": repr(e)}
+        line["also"] = also
+    if solo and not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(w, k)
+        line["cpu_baseline_single_thread"] = cpu_baseline_single_thread(args.config)
     if rank == 0:
         print(json.dumps(line))
-    if dist:
-        dist.close()
+    if group:
+        group.close()
     return 0
 
 

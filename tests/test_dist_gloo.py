@@ -58,3 +58,23 @@ def test_two_gloo_ranks(tmp_path):
     assert outs[0]["shard"] == [0, 4] and outs[1]["shard"] == [4, 7]
     assert outs[0]["agree"] and outs[1]["agree"]
     assert outs[0]["pages"] > 0 and outs[1]["pages"] > 0
+
+
+def test_bench_starts_its_own_ranks():
+    """`python bench.py --gpus 2` without torchrun starts two ranks itself (torch.distributed.run,
+    rendezvous on 127.0.0.1).  On a CPU machine the host leg of the path (--impl host-plan: plan
+    compilation only, gloo) runs through exactly the launch, sharding, barrier and
+    max-over-ranks code the GPU arm uses."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "host-plan",
+                          "--config", "c2", "--steps", "4", "--warmup", "3"], env=env, capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                     # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["impl"] == "host-plan" and line["scaling"] == "weak"
+    assert line["config"]["sequences_per_rank"] == 8           # shard_units: one batch of 8 per rank
+    # all ranks' units / the slowest rank's time
+    assert abs(line["value"] - 2 * 8 * 4 / (line["ms_per_step"] * 4e-3)) < 1e-6 * line["value"]
