@@ -710,6 +710,8 @@ def self_launch(args):
 
 
 def measure(name, args, dev, seed, group, world, layers=None, want_e2e=True, want_extras=False):
+    if args.lean:
+        want_e2e = want_extras = False
     """One configuration: device-resident cycle timing (exactly args.steps cycles, then the
     per-step statistics), optionally e2e and the side calls.  Returns (result dict, Cycle)."""
     import torch
@@ -720,7 +722,8 @@ def measure(name, args, dev, seed, group, world, layers=None, want_e2e=True, wan
         group.barrier()
     torch.cuda.synchronize()
     with ClockSampler(int(dev.split(":")[1])) as clocks:
-        total_ms, dec_ms, ver_ms, stats = cy.time_steps(args.steps, max(3, args.warmup))
+        total_ms, dec_ms, ver_ms, stats = cy.time_steps(args.steps, max(3, args.warmup),
+                                                        *((0, 0.0) if args.lean else ()))
     torch.cuda.synchronize()
     local_ms = total_ms
     if group:
@@ -820,6 +823,9 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the other configurations")
     ap.add_argument("--sweep-layers", type=int, default=None, help="layer count of the side configurations")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline legs")
+    ap.add_argument("--lean", action="store_true",
+                    help="only the --steps timed cycles: no extra replays for the statistics, no e2e, no side "
+                         "calls (for runs under a profiler, which should launch as little as possible)")
     ap.add_argument("--oracle-sample", type=float, default=0.0, help=argparse.SUPPRESS)
     ap.add_argument("--max-cluster", type=int, default=-1)
     ap.add_argument("--ring-slots", type=int, default=-1)
@@ -870,7 +876,7 @@ def main():
                                                  "pdl": args.pdl, "max_cluster": args.max_cluster, "ring_slots": args.ring_slots,
                                                  "ctas_per_sm": args.ctas_per_sm, "early_kv": args.early_kv,
                                                  "kv_layout": args.kv_layout}),
-        "clocks": res["clocks"], "per_step": res["per_step"], "e2e": res["e2e"],
+        "clocks": res["clocks"], "per_step": res["per_step"], "e2e": res.get("e2e"),
         "gpu_launches": res["gpu_launches"],
         "roofline": res[dominant], "roofline_decode": res["decode"], "roofline_verify": res["verify"],
         "us_per_layer_decode": res["us_per_layer_decode"],
@@ -883,7 +889,7 @@ def main():
             line[key] = res[key]
     cy.free()
 
-    if solo and not args.no_sweep:
+    if solo and not args.no_sweep and not args.lean:
         also = {}
         plan = [n for n in ("c4", "c3", "c2", "c5") if n != args.config]
         for name in plan:
@@ -905,7 +911,7 @@ def main():
         except Exception as e:
             also["c1"] = {"error": repr(e)}
         line["also"] = also
-    if solo and not args.no_cpu:
+    if solo and not args.no_cpu and not args.lean:
         line["cpu_baseline"] = cpu_baseline(w, k)
         line["cpu_baseline_single_thread"] = cpu_baseline_single_thread(args.config)
     if rank == 0:
