@@ -512,7 +512,10 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
 #pragma unroll
     for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     float m_run[2] = {-INFINITY, -INFINITY};                 // running max (log2 units)
-    float l_run[2] = {0.f, 0.f};                             // this lane's share of the row sums
+    // Row sums of the rounded weights: one more MMA per page, P times a matrix of ones, gives every
+    // thread the complete sum of its two rows (the same fp32 sum of the same bf16 weights that the
+    // P V product uses, so out = sum(p v) / sum(p) stays a true weighted mean).
+    float l_acc[4] = {0.f, 0.f, 0.f, 0.f};                   // [0] row gid, [2] row gid + 8
     const float sc = p.scale_log2;
     const int full_vis_limit = L - item.n_q;                 // tokens <= this are visible to all rows
 
@@ -521,14 +524,24 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     const int lm = lane >> 3, lr = lane & 7;
     const int k_tok = ((lm >> 1) << 3) + lr, k_cbit = lm & 1;   // K: matrices (n-tile, k-half)
     const int v_tok = ((lm & 1) << 3) + lr, v_cbit = lm >> 1;   // V^T: matrices (k-half, n-tile)
+    // Byte offset of this lane's ldmatrix row inside a tile for 16-byte chunk pair c (c = 0, 2, 4, 6):
+    // row * 128 + (((c + cbit) ^ lr) << 4).  c is even and cbit is one bit, so (c + cbit) ^ lr
+    // = c ^ (cbit ^ lr): the lane's part is a constant and the chunk pair enters as one XOR.
+    const uint32_t k_lane_off = (uint32_t)(k_tok * 128 + ((k_cbit ^ lr) << 4));
+    const uint32_t v_lane_off = (uint32_t)(v_tok * 128 + ((v_cbit ^ lr) << 4));
+    const uint32_t ones_bf16 = 0x3F803F80u;                    // two bf16 1.0: B operand of the row-sum MMA
 
+    // the group's ring position and barrier phase advance by counting: depth is a run-time value
+    // and a division per page would cost more than the page's address arithmetic
+    int ring_pos = 0;
+    uint32_t parity = 0;
     for (int i = 0;; ++i) {
-        const int s = grp * depth + i % depth;
-        const uint32_t parity = (i / depth) & 1;
-        mbar_wait(smem_u32(&tail->full[s]), parity, deadline, &tail->timed_out);
+        const int s = grp * depth + ring_pos;
+        const bool arrived = mbar_wait(smem_u32(&tail->full[s]), parity, deadline, &tail->timed_out);
         if (i == 0) KAP_TRACE_POINT(blockIdx.x, 3);
         const int page = tail->slot_page[s];
-        if (page < 0 || tail->timed_out) break;              // the list is exhausted
+        if (page < 0 || !arrived) break;                     // the list is exhausted (or a wait ran out)
+        if (++ring_pos == depth) { ring_pos = 0; parity ^= 1u; }
         const uint32_t tmask = kPlain ? 0xFFFFu : id_mask[page];
         const uint32_t kb = smem_u32(ring + s * kPageHeadBytes);
         const uint32_t vb = kb + kTileBytes;
@@ -539,8 +552,7 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             uint32_t b0, b1, b2, b3;
-            ldsm_x4(kb + (ks >> 2) * kHalfTileBytes + k_tok * 128
-                       + ((((ks & 3) * 2 + k_cbit) ^ lr) << 4), b0, b1, b2, b3);
+            ldsm_x4(((kb + k_lane_off) ^ (uint32_t)((ks & 3) << 5)) + (ks >> 2) * kHalfTileBytes, b0, b1, b2, b3);
             mma_bf16(sacc[0], qf[ks], b0, b1);
             mma_bf16(sacc[1], qf[ks], b2, b3);
         }
@@ -586,24 +598,21 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
         pa[1] = pack_bf16(ex2(fmaf(sacc[0][2], sc, -mu[1])), ex2(fmaf(sacc[0][3], sc, -mu[1])));
         pa[2] = pack_bf16(ex2(fmaf(sacc[1][0], sc, -mu[0])), ex2(fmaf(sacc[1][1], sc, -mu[0])));
         pa[3] = pack_bf16(ex2(fmaf(sacc[1][2], sc, -mu[1])), ex2(fmaf(sacc[1][3], sc, -mu[1])));
-        // the row sums use the rounded weights, so out = sum(p v) / sum(p) is a true average
-        l_run[0] = fmaf(l_run[0], corr[0],
-                        (bf16_lo(pa[0]) + bf16_hi(pa[0])) + (bf16_lo(pa[2]) + bf16_hi(pa[2])));
-        l_run[1] = fmaf(l_run[1], corr[1],
-                        (bf16_lo(pa[1]) + bf16_hi(pa[1])) + (bf16_lo(pa[3]) + bf16_hi(pa[3])));
         if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
                 o[n][0] *= corr[0]; o[n][1] *= corr[0];
                 o[n][2] *= corr[1]; o[n][3] *= corr[1];
             }
+            l_acc[0] *= corr[0]; l_acc[1] *= corr[0];
+            l_acc[2] *= corr[1]; l_acc[3] *= corr[1];
         }
+        mma_bf16(l_acc, pa, ones_bf16, ones_bf16);
         // O += P V   (16 n-tiles of 8 output columns, two per ldmatrix)
 #pragma unroll
         for (int n2 = 0; n2 < 8; ++n2) {
             uint32_t v0, v1, v2, v3;
-            ldsm_x4_t(vb + (n2 >> 2) * kHalfTileBytes + v_tok * 128
-                         + ((((n2 & 3) * 2 + v_cbit) ^ lr) << 4), v0, v1, v2, v3);
+            ldsm_x4_t(((vb + v_lane_off) ^ (uint32_t)((n2 & 3) << 5)) + (n2 >> 2) * kHalfTileBytes, v0, v1, v2, v3);
             mma_bf16(o[2 * n2], pa, v0, v1);
             mma_bf16(o[2 * n2 + 1], pa, v2, v3);
         }
@@ -628,11 +637,7 @@ kap_attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPara
     KAP_TRACE_POINT(blockIdx.x, 4);
 
     // ------------------------------------------------ combine the four warps' states, write out
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 1);
-        l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 2);
-    }
+    const float l_run[2] = {l_acc[0], l_acc[2]};       // complete row sums (every column of P x ones)
     __syncthreads();                                   // all tile reads done: the ring is scratch now
     float* scratch = reinterpret_cast<float*>(ring) + warp * (kRowTile * kScratchStride);
 #pragma unroll

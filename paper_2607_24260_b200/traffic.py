@@ -1,8 +1,11 @@
 """DRAM traffic of the attention kernel per algorithmic byte, as measured by one ncu capture, kept in
 a small tracked text file together with a digest of the kernel sources it was measured on.
 
-    python -m paper_2607_24260_b200.traffic decode <ncu raw csv> <algorithmic bytes per launch>
-    python -m paper_2607_24260_b200.traffic verify <ncu raw csv> <algorithmic bytes per launch>
+    python -m paper_2607_24260_b200.traffic decode <ncu raw csv> <algorithmic bytes per launch> [kernel name part]
+    python -m paper_2607_24260_b200.traffic verify <ncu raw csv> <algorithmic bytes per launch> [kernel name part]
+
+(kernel name part: which launches of the csv to average, e.g. "split_kernel<1" for the proposal
+instantiation and "split_kernel<2" for the verification one; default: every kap_attn_split_kernel.)
 
 The csv is what `ncu -i <report> --page raw --csv` prints for a capture of kap_attn_split_kernel
 (`dram__bytes_read.sum` and `dram__bytes_write.sum` per launch).  The benchmark reads the file
@@ -86,6 +89,6 @@ def write_ratio(kind: str, ratio: float, note: str):
 if __name__ == "__main__":
     kind, path, alg = sys.argv[1], sys.argv[2], float(sys.argv[3])
     assert kind in ("decode", "verify")
-    t = traffic_from_csv(path)
+    t = traffic_from_csv(path, *sys.argv[4:5])
     write_ratio(kind, t / alg, f"{t:.0f}B/{alg:.0f}B from {os.path.basename(path)}")
     print(kind, t / alg)
