@@ -627,7 +627,8 @@ def cpu_baseline_single_thread(config, budget_s=6.0):
 def run_reference(args):
     """--impl reference: the CPU oracle on the same metric and workload (rank 0 only; the other
     ranks exit without work).  Each step times a bounded sample of (sequence, layer) units, sized
-    so that warm-up + steps end within about two and a half minutes of oracle work."""
+    so that warm-up + steps end within about a hundred seconds of oracle work (plus the host-side
+    generation of one layer of KV)."""
     rank, _, world = dist_env()
     if rank != 0:
         return 0
@@ -635,7 +636,7 @@ def run_reference(args):
     w = synth.CONFIGS[args.config](0)
     k = int(w.n_q.max())
     sm = OracleSampler(w)
-    per_step = 150.0 / max(1, args.steps + args.warmup)
+    per_step = 100.0 / max(1, args.steps + args.warmup)
     t_unit = sm.run_units(1)                              # calibration
     cycles, units_per_step = [], max(1, int(per_step / max(t_unit, 1e-6)))
     for i in range(args.warmup + args.steps):
