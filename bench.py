@@ -711,11 +711,11 @@ def self_launch(args):
 
 
 def measure(name, args, dev, seed, group, world, layers=None, want_e2e=True, want_extras=False):
-    if args.lean:
-        want_e2e = want_extras = False
     """One configuration: device-resident cycle timing (exactly args.steps cycles, then the
     per-step statistics), optionally e2e and the side calls.  Returns (result dict, Cycle)."""
     import torch
+    if args.lean:
+        want_e2e = want_extras = False
     cy = Cycle(name, seed=seed, layers=layers, device=dev, kv_layout=args.kv_layout,
                decode_chunk=args.decode_chunk, verify_chunk=args.verify_chunk)
     cy.capture()
@@ -749,7 +749,8 @@ def measure(name, args, dev, seed, group, world, layers=None, want_e2e=True, wan
                               "device-resident state"}
     cy.ws_d.check()
     cy.ws_v.check()
-    res["gpu_launches"] = cy.launches_per_step * stats["replays"]
+    res["gpu_launches"] = cy.launches_per_step * args.steps          # inside the timed region of `value`
+    res["per_step"]["gpu_launches_incl_statistics_replays"] = cy.launches_per_step * stats["replays"]
     if want_extras:
         res["other_calls"] = time_extras(cy)
         from paper_2607_24260_b200 import kap

@@ -428,3 +428,53 @@ def test_out_of_range_page_is_reported_not_dereferenced():
     # the context is still usable and the status word was cleared
     good = gu.run_decode(_decode_rows(w, q_bits), pool, plan, w.ctx_len)
     _check_pair(good, gu.oracle_decode(_decode_rows(w, q_bits), pool_bits, plan, w.ctx_len), "after error")
+
+
+def test_failed_schedule_leaves_the_previous_one_in_force():
+    """A kap_schedule call that fails (more rows than the workspace holds; a changed ring size on
+    top, which a half-applied update would have kept) changes nothing: the attention call that
+    follows runs on the previous schedule and still matches the oracle."""
+    w = synth.config2(3, batch=2, L=3000, layers=1)
+    q_bits, pool_bits, pool = _workload_case(w, 3)
+    plan = kap.compile_workload(w)
+    ws = kap.Workspace(max_rows_per_item=4, max_batch=2)
+    first = ws.schedule(np.diff(plan["plan_indptr"]), None, 32, 8)
+    kap.set_launch_options(-1, -1, -1, -1, 12)               # another ring size for the next schedule
+    try:
+        with pytest.raises(kap.KapError) as e:
+            ws.schedule(np.diff(plan["plan_indptr"]), [8, 8], 32, 8)      # 32 rows > 4
+        assert e.value.code == kap.ERR_CAPACITY
+    finally:
+        kap.set_launch_options(-1, -1, -1, -1, 8)
+    assert ws.info() == first
+    qd = gu.bits_to_dev(_decode_rows(w, q_bits))
+    out = torch.full_like(qd, float("nan"))
+    kap.selected_decode_attn(qd, pool, gu.i32(plan["plan_indptr"]), gu.i32(plan["plan_phys_pages"]),
+                             gu.i32(plan["plan_logical_pages"]), gu.i32(w.ctx_len), out, ws)
+    ws.check()
+    ref = gu.oracle_decode(_decode_rows(w, q_bits), pool_bits, plan, w.ctx_len)
+    assert_close(gu.dev_bf16_to_f64(out), ref[0], what="decode on the schedule that stayed in force")
+    ws.close()
+
+
+def test_workspace_calls_keep_the_callers_device_and_attention_checks_it():
+    """kap_workspace_create / kap_schedule put the calling thread's current device back; an
+    attention call made while another device is current is refused (one-GPU machines: only the first
+    half can run)."""
+    before = torch.cuda.current_device()
+    ws = kap.Workspace(device=0, max_rows_per_item=4, max_batch=1)
+    ws.schedule([8], None, 32, 8)
+    assert torch.cuda.current_device() == before
+    if torch.cuda.device_count() > 1:
+        w = synth.config2(0, batch=1, L=128, layers=1)
+        q_bits, pool_bits, pool = _workload_case(w, 1)
+        plan = kap.compile_workload(w)
+        ws.schedule(np.diff(plan["plan_indptr"]), None, 32, 8)
+        qd = gu.bits_to_dev(_decode_rows(w, q_bits))
+        out = torch.zeros_like(qd)
+        with torch.cuda.device(1):
+            with pytest.raises(kap.KapError) as e:
+                kap.selected_decode_attn(qd, pool, gu.i32(plan["plan_indptr"]), gu.i32(plan["plan_phys_pages"]),
+                                         gu.i32(plan["plan_logical_pages"]), gu.i32(w.ctx_len), out, ws)
+            assert e.value.code == kap.ERR_INVALID_ARG
+    ws.close()
