@@ -776,6 +776,100 @@ def side_entry(r, cy):
     return out
 
 
+class TwoMicroBatches(Cycle):
+    """The same configuration run as two micro-batches (first and second half of the sequences) on
+    two streams, each an independent chain over the layers - what a serving engine does when it
+    interleaves two micro-batches of one forward pass.  The kernels, plans and pool are the same;
+    only the launch structure differs: while one chain's launch ramps up, drains or sits at a
+    kernel boundary, the other one streams.  A side measurement: it shows what the per-launch
+    fixed costs of the single chain cost, it is not the headline."""
+
+    def __init__(self, name, seed, layers=None, device="cuda:0", max_cluster=16, ctas_per_sm=0, restore_max_cluster=16):
+        super().__init__(name, seed, layers=layers, device=device)
+        torch, kap, w = self.torch, self.kap, self.w
+        B, Hq, Hkv = w.batch, w.num_q_heads, w.num_kv_heads
+        assert B % 2 == 0
+        i32 = lambda a: torch.from_numpy(np.array(a, dtype=np.int32)).to(device)
+        self.side = torch.cuda.Stream(device=device)
+        self.halves = []
+        kap.set_launch_options(-1, -1, ctas_per_sm, max_cluster, -1)     # two launches share the SMs' CTA slots
+        try:
+            for lo, hi in ((0, B // 2), (B // 2, B)):
+                pi, bi = self.plan["plan_indptr"], w.bt_indptr
+                h = {"lo": lo, "hi": hi, "rows": (int(w.q_indptr[lo]), int(w.q_indptr[hi])),
+                     "plan_indptr": i32(pi[lo:hi + 1] - pi[lo]),
+                     "plan_phys": i32(self.plan["plan_phys_pages"][pi[lo]:pi[hi]]),
+                     "plan_logical": i32(self.plan["plan_logical_pages"][pi[lo]:pi[hi]]),
+                     "ctx": i32(w.ctx_len[lo:hi]), "q_indptr": i32(w.q_indptr[lo:hi + 1] - w.q_indptr[lo]),
+                     "bt_indptr": i32(bi[lo:hi + 1] - bi[lo]), "bt_pages": i32(w.bt_pages[bi[lo]:bi[hi]])}
+                dev_index = int(device.split(":")[1])
+                h["ws_d"] = kap.Workspace(dev_index, 8192, Hq // Hkv, hi - lo)
+                h["ws_v"] = kap.Workspace(dev_index, 8192, int(w.n_q.max()) * (Hq // Hkv), hi - lo)
+                h["info_d"] = h["ws_d"].schedule(self.n_sel[lo:hi], None, Hq, Hkv)
+                h["info_v"] = h["ws_v"].schedule(self.n_pages[lo:hi], w.n_q[lo:hi], Hq, Hkv)
+                self.halves.append(h)
+        finally:
+            kap.set_launch_options(-1, -1, 0, restore_max_cluster, -1)
+        self.info_d = [h["info_d"] for h in self.halves]
+        self.info_v = [h["info_v"] for h in self.halves]
+
+    def _fork(self, body):
+        torch = self.torch
+        cur = torch.cuda.current_stream()
+        self.side.wait_stream(cur)
+        for h, st in zip(self.halves, (cur, self.side)):
+            with torch.cuda.stream(st):
+                body(h)
+        cur.wait_stream(self.side)
+
+    def enqueue_proposal(self):
+        kap = self.kap
+
+        def body(h):
+            for step in range(self.k):
+                for layer in range(self.layers):
+                    kap.selected_decode_attn(self.q_dec[step, layer, h["lo"]:h["hi"]], self.pool_attn[layer],
+                                             h["plan_indptr"], h["plan_phys"], h["plan_logical"], h["ctx"],
+                                             self.out_dec[step, layer, h["lo"]:h["hi"]], h["ws_d"])
+        self._fork(body)
+
+    def enqueue_verify(self):
+        kap = self.kap
+
+        def body(h):
+            r0, r1 = h["rows"]
+            for layer in range(self.layers):
+                kap.verify_attn(self.q_ver[layer, r0:r1], h["q_indptr"], self.pool_attn[layer], h["bt_indptr"],
+                                h["bt_pages"], h["ctx"], self.out_ver[layer, r0:r1], h["ws_v"])
+        self._fork(body)
+
+    def free(self):
+        for h in self.halves:
+            h["ws_d"].check(); h["ws_v"].check()
+            h["ws_d"].close(); h["ws_v"].close()
+        super().free()
+
+
+def time_two_microbatches(name, args, dev, layers):
+    import torch
+    cy = TwoMicroBatches(name, seed=0, layers=layers, device=dev,
+                         restore_max_cluster=args.max_cluster if args.max_cluster > 0 else 16)
+    cy.capture()
+    total_ms, dec_ms, ver_ms, stats = cy.time_steps(args.steps, max(3, args.warmup))
+    r = summarise(cy, args.steps, total_ms, dec_ms, ver_ms)
+    out = {"workload": cy.w.note, "layers_timed": cy.layers, "replays": stats["replays"],
+           "note": "two micro-batches (half of the sequences each) on two streams, each an independent chain of "
+                   "layers; same kernels, plans and pool as the headline; per layer = both micro-batches",
+           "us_per_layer_decode": r["us_per_layer_decode"], "us_per_layer_verify": r["us_per_layer_verify"],
+           "us_per_layer_decode_median_best": [round(stats["us_per_layer_decode"][x], 3) for x in ("median", "best")],
+           "us_per_layer_verify_median_best": [round(stats["us_per_layer_verify"][x], 3) for x in ("median", "best")],
+           "decode_frac_of_measured": r["decode"]["frac"], "decode_frac_of_8TBs": r["decode"]["frac_of_nominal_8TBs"],
+           "verify_frac_of_measured": r["verify"]["frac"], "verify_frac_of_8TBs": r["verify"]["frac_of_nominal_8TBs"],
+           "tokens_per_s": r["tokens_per_s"], "schedule": r["schedule"]}
+    cy.free()
+    return out
+
+
 def time_c1_warm_cold(args, dev):
     """Configuration 1 (one sequence, one layer, 4096 tokens): its 16.8 MB of KV stay in the L2
     between replays, so one proposal pass and the verification pass are timed twice - replayed
@@ -899,15 +993,18 @@ def main():
                 full = name in ("c3", "c4")                  # measured like the headline: e2e and CPU baseline too
                 layers = args.sweep_layers if args.sweep_layers else (None if name != "c5" else 4)
                 r, c2 = measure(name, args, dev, 0, None, 1, layers=layers, want_e2e=full)
-                if full and not args.no_cpu:
+                if full and not args.no_cpu:          # all cores; the one-thread figure is the headline's only
                     r["cpu_baseline"] = cpu_baseline(c2.w, c2.k)
-                    r["cpu_baseline_single_thread"] = cpu_baseline_single_thread(name)
                 if full:
                     r["roofline_decode"], r["roofline_verify"] = r["decode"], r["verify"]
                 also[name] = side_entry(r, c2)
                 c2.free()
             except Exception as e:       # a side measurement must not lose the main line
                 also[name] = {"error": repr(e)}
+        try:       # the headline configuration once more, as two interleaved micro-batches (8 layers)
+            also[args.config + "_two_microbatches"] = time_two_microbatches(args.config, args, dev, 8)
+        except Exception as e:
+            also[args.config + "_two_microbatches"] = {"error": repr(e)}
         try:
             also["c1"] = time_c1_warm_cold(args, dev)
         except Exception as e:
