@@ -18,7 +18,8 @@ persistent state and stays on the device).
 
 The headline workload is configuration 4 (B = 4, 128K context, all 32 layers, 68.7 GB of KV: the
 largest single-GPU configuration, inside the 32K-128K range the target is stated on);
-configuration 3 is measured beside it in full, configurations 2, 5 and 1 as side lines.
+configuration 3 is measured beside it in full, configurations 2 (32 layers), 5 (16 layers) and 1 as
+side lines.
 
 N > 1: one process per GPU, every rank runs its own batch (weak scaling, no data-path
 collective); time = max over ranks.  Under torchrun the ranks come from the environment; a plain
@@ -991,7 +992,7 @@ def main():
         for name in plan:
             try:
                 full = name in ("c3", "c4")                  # measured like the headline: e2e and CPU baseline too
-                layers = args.sweep_layers if args.sweep_layers else (None if name != "c5" else 4)
+                layers = args.sweep_layers if args.sweep_layers else None    # each at its own full layer count
                 r, c2 = measure(name, args, dev, 0, None, 1, layers=layers, want_e2e=full)
                 if full and not args.no_cpu:          # all cores; the one-thread figure is the headline's only
                     r["cpu_baseline"] = cpu_baseline(c2.w, c2.k)
