@@ -506,6 +506,14 @@ def phase_report(kap, k, t_sel, t_verify, t_full):
         m = kap.phase_model(k, h, min(s_time, 1.0), 0.0, 0.0, t_full)
         rep[f"model_speedup_h{h}"] = m["speedup"]                       # verifier at t_full (Eq. 7)
         rep[f"measured_speedup_h{h}"] = (1 + k * h) * t_full / (k * t_sel + t_verify)
+    # the fallback controller on the same profiled costs (Section 4.2): what it would decide for a
+    # request whose observed Top-3 acceptance is h (1000 verified proposals, attention-only costs)
+    verdicts = {}
+    for h in (0.02, 0.05, 0.10, 0.50, 0.95):
+        d = kap.fallback_decide([int(round(1000 * h))], [1000], [s_time], [t_full], h_min=0.0, s_max=1.0)
+        verdicts[f"h={h}"] = {"force_full": int(d["force_full"][0]), "reasons": int(d["reasons"][0]),
+                              "slack_us": float(d["slack"][0]), "budget_scale": float(d["budget_scale"][0])}
+    rep["fallback_controller"] = verdicts
     return rep
 
 
