@@ -253,12 +253,13 @@ class Workspace:
     def __init__(self, device=0, max_items=8192, max_rows_per_item=16, max_batch=256):
         self._h = C.c_void_p()
         self.device = int(device)
+        self._destroy = lib().kap_workspace_destroy
         _check(lib().kap_workspace_create(C.byref(self._h), self.device, max_items,
                                           max_rows_per_item, max_batch))
 
     def close(self):
         if getattr(self, "_h", None) is not None and self._h:
-            lib().kap_workspace_destroy(self._h)
+            self._destroy(self._h)           # bound at construction: module globals may be gone at exit
             self._h = None
 
     __del__ = close
