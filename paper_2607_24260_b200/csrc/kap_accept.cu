@@ -51,6 +51,24 @@ __device__ __forceinline__ void push(Top3& t, Key x) {
     const Key b1 = max(t.k[1], r1), r2 = min(t.k[1], r1);
     t.k[0] = b0; t.k[1] = b1; t.k[2] = max(t.k[2], r2);
 }
+// The best three keys held anywhere in the warp, left in every lane (each lane passes its own best
+// three, sorted).  Three rounds of "largest head key in the warp; its owner moves on to its next
+// one": keys are unique (the index is part of them), so exactly one lane advances per round, and a
+// 64-bit maximum is two 32-bit warp reductions - about a tenth of the instructions of a butterfly
+// of pairwise top-3 merges.
+__device__ __forceinline__ void warp_top3(Top3& t) {
+    Key out[3];
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const Key head = t.k[0];
+        const uint32_t hi = __reduce_max_sync(0xffffffffu, (uint32_t)(head >> 32));
+        const uint32_t lo = __reduce_max_sync(0xffffffffu, (uint32_t)(head >> 32) == hi ? (uint32_t)head : 0u);
+        const Key best = ((Key)hi << 32) | lo;
+        out[r] = best;
+        if (head == best && best != 0ull) { t.k[0] = t.k[1]; t.k[1] = t.k[2]; t.k[2] = 0ull; }
+    }
+    t.k[0] = out[0]; t.k[1] = out[1]; t.k[2] = out[2];
+}
 __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -108,14 +126,7 @@ kap_top3_rows_kernel(const float* __restrict__ logits, long long row_stride, int
     Top3 t;
     t.k[0] = as_key(sc.u0, sc.i0); t.k[1] = as_key(sc.u1, sc.i1); t.k[2] = as_key(sc.u2, sc.i2);
     // warp merge, then the 8 warps through shared memory
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        Key o[3];
-#pragma unroll
-        for (int k = 0; k < 3; ++k) o[k] = __shfl_xor_sync(0xffffffffu, t.k[k], off);
-#pragma unroll
-        for (int k = 0; k < 3; ++k) push(t, o[k]);
-    }
+    warp_top3(t);
     __shared__ Top3 part[kRowsThreads / 32];
     __shared__ Top3 peers[8];                       // first CTA only: the other CTAs' candidates land here
     if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = t;
@@ -124,21 +135,11 @@ kap_top3_rows_kernel(const float* __restrict__ logits, long long row_stride, int
     // initialised and every peer is running
     if (S > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     if (threadIdx.x >= 32) return;
-    // warp 0 merges the warps' candidates: lane w takes warp w's three, then a butterfly over 16 lanes
+    // warp 0 merges the warps' candidates: lane w takes warp w's three
     const int lane = threadIdx.x;
-    auto butterfly16 = [&](Top3& x) {
-#pragma unroll
-        for (int off = 8; off > 0; off >>= 1) {
-            Key o[3];
-#pragma unroll
-            for (int k = 0; k < 3; ++k) o[k] = __shfl_xor_sync(0xffffffffu, x.k[k], off);
-#pragma unroll
-            for (int k = 0; k < 3; ++k) push(x, o[k]);
-        }
-    };
     const int n_warps = (int)(blockDim.x >> 5);
     if (lane < n_warps) t = part[lane]; else t.k[0] = t.k[1] = t.k[2] = 0;
-    butterfly16(t);                                 // lanes 0..15 now all hold the CTA's best three
+    warp_top3(t);                                   // every lane now holds the CTA's best three
     if (S > 1 && part_id != 0) {
         // push this CTA's three candidates into the first CTA's shared memory and arrive on its
         // barrier (the arrive orders the stores before it); nobody reads this CTA's memory
@@ -174,7 +175,7 @@ kap_top3_rows_kernel(const float* __restrict__ logits, long long row_stride, int
         if (ok) {
             if (lane >= 1 && lane < S) t = peers[lane];
             else if (lane != 0) t.k[0] = t.k[1] = t.k[2] = 0;
-            butterfly16(t);                         // S <= 8 peers
+            warp_top3(t);                           // S <= 8 peers
         }
     }
     if (lane == 0) {
