@@ -569,6 +569,16 @@ kap_status kap_selected_decode_attn_static(
     int32_t* device_status,            /* DEVICE int32 or NULL */
     void* cuda_stream);
 
+/*
+ * kap_device_sm_rates - relative memory-streaming rate of every SM of a device (mean 1.0), measured
+ * once per process on first use (about a millisecond; allocates and frees a temporary buffer of
+ * 3 MiB per SM).  On B200 groups of 8 to 10 SMs share a fixed-bandwidth port towards L2 / HBM, so
+ * while all SMs stream an SM of a larger group is served up to 20 % slower; kap_schedule uses these
+ * rates to size the slices of full-context launches.  The paper has no counterpart.
+ * rates may be NULL (then only *n_sms is written).  Errors: KAP_ERR_CUDA, KAP_ERR_CAPACITY.
+ */
+kap_status kap_device_sm_rates(int32_t device, int32_t capacity, float* rates /* HOST out */, int32_t* n_sms);
+
 /* Synchronises `cuda_stream` and returns the device status word of the workspace (KAP_OK,
  * KAP_ERR_TIMEOUT or KAP_ERR_DEVICE_INDEX), clearing it. */
 kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);

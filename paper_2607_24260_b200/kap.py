@@ -60,6 +60,7 @@ SIGNATURES = {
                                       C.POINTER(C.c_double)]),
     "kap_materialize_view": (C.c_int, [_vp, C.c_int64, _vp, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                        _vp, C.c_int64, _vp, _vp, _vp]),
+    "kap_device_sm_rates": (C.c_int, [C.c_int32, C.c_int32, _f32p, _i32p]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
     "kap_set_launch_options": (C.c_int, [C.c_int32] * 5),
     "kap_launch_count": (C.c_int64, []),
@@ -390,6 +391,15 @@ def fallback_decide(accepted_sum, proposed_sum, s, kv, w_main=0.0, w_prop=0.0, m
         float(s_max), _ptr(flags, C.c_int32), _ptr(rt, C.c_int32), _ptr(conf, C.c_double),
         float(confidence_min), _ptr(out["force_full"], C.c_uint8), _ptr(out["reasons"], C.c_int32),
         _ptr(out["h"], C.c_double), _ptr(out["slack"], C.c_double), _ptr(out["budget_scale"], C.c_double)))
+    return out
+
+
+def device_sm_rates(device=0):
+    """kap_device_sm_rates: numpy array of the relative streaming rate of every SM (mean 1)."""
+    n = C.c_int32(0)
+    _check(lib().kap_device_sm_rates(int(device), 0, None, C.byref(n)))
+    out = np.zeros(n.value, dtype=np.float32)
+    _check(lib().kap_device_sm_rates(int(device), n.value, _ptr(out, C.c_float), C.byref(n)))
     return out
 
 
