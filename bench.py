@@ -912,6 +912,29 @@ def time_c1_warm_cold(args, dev):
                    "cold = 512 MB streamed before every replay; launch-latency bound, not a bandwidth figure"}
     for mode in ("warm", "cold"):
         out[mode] = {"decode_us": timed(g1, mode == "cold"), "verify_us": timed(cy.graph_v, mode == "cold")}
+
+    def chained(enqueue, n=32):
+        """Device time per pass when n passes sit in ONE graph (no host launch between them): what
+        the pass costs the GPU itself.  The passes read the same L2-resident KV."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(n):
+                enqueue()
+        t = []
+        for i in range(3 + 10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); g.replay(); e1.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                t.append(e0.elapsed_time(e1) / n * 1e3)
+        return [round(statistics.median(t), 2), round(min(t), 2)]
+
+    one_decode = lambda: cy.kap.selected_decode_attn(cy.q_dec[0, 0], cy.pool_attn[0], cy.d_plan_indptr, cy.d_plan_phys,
+                                                     cy.d_plan_logical, cy.d_ctx, cy.out_dec[0, 0], cy.ws_d)
+    one_verify = lambda: cy.kap.verify_attn(cy.q_ver[0], cy.d_q_indptr, cy.pool_attn[0], cy.d_bt_indptr, cy.d_bt_pages,
+                                            cy.d_ctx, cy.out_ver[0], cy.ws_v)
+    out["warm_chained"] = {"decode_us": chained(one_decode), "verify_us": chained(one_verify),
+                           "note": "32 passes in one graph, per pass: without the host's launch latency"}
     del flush
     cy.free()
     return out

@@ -35,6 +35,7 @@ int64_t chunks_for(const int32_t* len, int32_t batch, int32_t hkv, int64_t t) {
 // that when the kernel can use its push-style reduction, i.e. for items of at most 4 query rows).
 constexpr int64_t kFixedPages = 6;                        // + rows / 2: wider items start and end slower
 constexpr int64_t kMergePassPages = 9;
+constexpr int64_t kMergeBatchPages = 3;                   // per further batch of 16 partial states of one list
 constexpr int64_t kLaterWavePages = 40;
 constexpr int64_t kClusterPagesX5 = 8;                    // per CTA of a cluster, in fifths of a page
 constexpr int64_t kPushClusterPagesX5 = 4;                // same, when the kernel reduces by pushing (<= 4 rows)
@@ -107,11 +108,12 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
         // per-CTA chunk of each item, longest first
         sizes.clear();
         bool merge_pass = false;
-        int64_t total = 0, longest = 0;
+        int64_t total = 0, longest = 0, most_splits = 1;
         for (int32_t b = 0; b < batch; ++b) {
             const int64_t n = splits[b], base = list_len[b] / n, rem = list_len[b] % n;
             if ((base + (rem ? 1 : 0) + C - 1) / C > cap) return;
             merge_pass |= n > 1;
+            most_splits = std::max(most_splits, n);
             for (int64_t i = 0; i < n; ++i) {
                 const int64_t sz = (base + (i < rem ? 1 : 0) + C - 1) / C + fixed;
                 for (int32_t g = 0; g < num_kv_heads; ++g) sizes.push_back(sz);
@@ -120,7 +122,8 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
             }
         }
         if ((int64_t)sizes.size() > item_cap) return;
-        const int64_t penalty = (merge_pass ? kMergePassPages : 0) + (C > 1 ? ((rows <= 4 ? kPushClusterPagesX5 : kClusterPagesX5) * C + 4) / 5 : 0);
+        // (the merge pass reads a list's partial states sixteen at a time, one memory round trip each)
+        const int64_t penalty = (merge_pass ? kMergePassPages + kMergeBatchPages * ((most_splits - 1) / 16) : 0) + (C > 1 ? ((rows <= 4 ? kPushClusterPagesX5 : kClusterPagesX5) * C + 4) / 5 : 0);
         if (std::max(longest, (total + slots - 1) / slots) + penalty >= best_cost) return;   // lower bound
         int64_t makespan = longest;
         if ((int64_t)sizes.size() > slots) {
@@ -138,13 +141,17 @@ kap_status build_schedule(int32_t batch, const int32_t* list_len, const int32_t*
         }
         if (makespan + penalty < best_cost) { best_cost = makespan + penalty; best_c = (int32_t)C; best_splits = splits; }
     };
-    static const int64_t kWaves[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 24, 32, 48, 64, INT32_MAX};
+    static const int64_t kWaves[] = {-1, 0, 1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 24, 32, 48, 64, INT32_MAX};
     for (int ci = 0; ci < kMaxCluster; ++ci) {
         const int64_t C = ci + 1, slots = cluster_slots[ci];
         if (slots <= 0) continue;
         int64_t last_budget = -1;
         for (int64_t waves : kWaves) {                       // the last entry: as many items as allowed
-            const int64_t budget = std::min<int64_t>(item_cap, waves == 1 ? std::min<int64_t>(slots, one_wave_slots[ci]) : slots * waves);
+            // (entries <= 0: a launch that fills only a half or a quarter of a wave - short lists are
+            // not worth a CTA per page and a merge pass over dozens of partial states)
+            const int64_t one_wave = std::min<int64_t>(slots, one_wave_slots[ci]);
+            const int64_t budget = std::min<int64_t>(item_cap, waves == -1 ? std::max<int64_t>(one_wave / 4, 1) : waves == 0 ? std::max<int64_t>(one_wave / 2, 1)
+                                                               : waves == 1 ? one_wave : slots * waves);
             if (budget == last_budget) break;
             last_budget = budget;
             const int64_t t = min_chunk(budget);
