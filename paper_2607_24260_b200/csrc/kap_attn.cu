@@ -74,6 +74,8 @@ std::atomic<int> g_max_cluster{kMaxCluster};       // largest thread-block clust
 std::atomic<int> g_early_kv{1};
 std::atomic<int> g_ring_slots{kDefaultSlots};
 std::atomic<int> g_ctas_per_sm{0};       // 0 = as many as fit (occupancy)
+constexpr int kWideMergeSplits = 24;     // partial states per list from which the wide merge kernel pays off ...
+constexpr int64_t kWideMergeRows = 1024; // ... as long as (lists x query rows) stays below this
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -249,7 +251,14 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
         cfg.dynamicSmemBytes = 0;
         cfg.numAttrs = n_pdl_attr;
         const MergeGroup* mg = ws->d_merge;
-        KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_merge_kernel, p, mg));
+        // eight threads per output cell when the lists have many partial states and the cells are
+        // few enough for that many blocks to be cheap
+        if (ws->max_splits >= kWideMergeSplits && (int64_t)ws->n_merge_groups * rows <= kWideMergeRows) {
+            cfg.gridDim = dim3((unsigned)ws->n_merge_groups, (unsigned)(2 * rows));
+            KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_merge_wide_kernel, p, mg));
+        } else {
+            KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_merge_kernel, p, mg));
+        }
         g_launches.fetch_add(1);
     }
     return KAP_OK;
@@ -412,7 +421,9 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     int32_t n_merge = 0;
     int64_t total_rows = 0;
     for (int32_t b = 0; b < batch; ++b) total_rows += n_q ? n_q[b] : 1;
+    int32_t max_splits = 1;
     for (size_t i = 0; i < groups.size(); ++i) {
+        max_splits = std::max(max_splits, groups[i].n_splits);
         ws->h_groups[i] = groups[i];
         if (groups[i].n_splits > 1) ws->h_merge[n_merge++] = groups[i];
     }
@@ -431,7 +442,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     ws->batch = batch; ws->n_items = (int32_t)items.size(); ws->n_groups = (int32_t)groups.size();
     ws->n_merge_groups = n_merge; ws->max_chunk = max_chunk; ws->row_tiles = row_tiles;
     ws->num_q_heads = num_q_heads; ws->num_kv_heads = num_kv_heads; ws->has_nq = n_q != nullptr;
-    ws->total_rows = total_rows; ws->cluster_size = cluster;
+    ws->total_rows = total_rows; ws->cluster_size = cluster; ws->max_splits = max_splits;
     int32_t mq = 1;
     for (int32_t b = 0; b < batch; ++b) mq = std::max(mq, n_q ? n_q[b] : 1);
     ws->max_nq = mq;

@@ -784,4 +784,52 @@ kap_attn_merge_kernel(const AttnParams p, const MergeGroup* merge_groups)
     KAP_TRACE_POINT(4096 + blockIdx.x, 5);
 }
 
+// The merge pass for lists with many partial states (one long sequence cut into 50 slices): the
+// next kernel on the stream waits for this pass, and one thread per output cell would read its
+// states in several dependent batches.  Here eight threads share a cell: thread j merges states
+// j, j + 8, ... (its loads all in flight together), then the eight running states are combined
+// pairwise in a fixed order, so results do not depend on timing.  grid.x = lists, grid.y = 2 x
+// query rows (a block = half a row of 32 four-column cells); a warp = 4 neighbouring cells x 8
+// state lanes.
+__global__ void __launch_bounds__(128)
+kap_attn_merge_wide_kernel(const AttnParams p, const MergeGroup* merge_groups)
+{
+    pdl_launch_dependents();
+    const MergeGroup g = merge_groups[blockIdx.x];          // static metadata: before the wait
+    const int64_t q_row0 = p.q_indptr ? p.q_indptr[g.seq] : g.seq;
+    const int R = blockIdx.y >> 1;
+    const int lane = threadIdx.x & 31, sl = lane >> 2;
+    const int c4 = (blockIdx.y & 1) * 16 + (threadIdx.x >> 5) * 4 + (lane & 3);
+    pdl_wait();
+    if (R >= g.n_q * p.G) return;                            // (the whole block: R is per block)
+    constexpr int kLanes = 8, kBatch = 8;
+    const int64_t base = (int64_t)g.first_item * p.rows_cap + R;
+    const int64_t stride = p.rows_cap;
+    Merged r; r.m = -INFINITY; r.l = 0.f; r.o = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i0 = 0; i0 < g.n_splits; i0 += kLanes * kBatch) {
+        float2 ml[kBatch];
+        float4 o[kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const int i = min(i0 + j * kLanes + sl, g.n_splits - 1);
+            ml[j] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + i * stride) * 2));
+            o[j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (base + i * stride) * kHeadDim) + c4);
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j)
+            if (i0 + j * kLanes + sl < g.n_splits) merge_into(r, ml[j].x, ml[j].y, o[j]);
+    }
+#pragma unroll
+    for (int d = 4; d < 32; d <<= 1) {                       // state lanes differ in lane bits 2..4
+        const float m2 = __shfl_xor_sync(0xffffffffu, r.m, d), l2 = __shfl_xor_sync(0xffffffffu, r.l, d);
+        float4 o2;
+        o2.x = __shfl_xor_sync(0xffffffffu, r.o.x, d); o2.y = __shfl_xor_sync(0xffffffffu, r.o.y, d);
+        o2.z = __shfl_xor_sync(0xffffffffu, r.o.z, d); o2.w = __shfl_xor_sync(0xffffffffu, r.o.w, d);
+        // both partners end with the same bits: the lower lane's state is always the left operand
+        if (lane & d) { Merged t; t.m = m2; t.l = l2; t.o = o2; merge_into(t, r.m, r.l, r.o); r = t; }
+        else merge_into(r, m2, l2, o2);
+    }
+    if (sl == 0) store_final(p, q_row0 + R / p.G, g.kv_head * p.G + R % p.G, c4, r);
+}
+
 }  // namespace kap

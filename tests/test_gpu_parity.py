@@ -303,11 +303,35 @@ def test_split_and_launch_option_invariance():
                     _check_pair(got, ref, f"pdl={pdl} early={early} cluster={cluster} chunk={chunk}")
                     # splits only reorder fp32 sums: far tighter than the oracle tolerance
                     np.testing.assert_allclose(got[0], one_split[0], atol=2e-3, rtol=1e-2)
-                    np.testing.assert_allclose(got[1], one_split[1], atol=1e-4)
+                    # (lse: the row sums are sums of bf16-rounded weights, and which way a weight rounds
+                    # depends on the slice's own running maximum: about 1e-4 between slicings)
+                    np.testing.assert_allclose(got[1], one_split[1], atol=3e-4)
                 got = gu.run_verify(q_bits, w.n_q, pool, w.bt_indptr, w.bt_pages, w.ctx_len)
                 _check_pair(got, ref_v, f"verify pdl={pdl} early={early} cluster={cluster}")
     finally:
         kap.set_launch_options(1, 1, 0, 16, 8)
+
+
+def test_one_long_sequence_many_partial_states():
+    """One sequence of 30 000 tokens: 8 lists cut into about 55 slices each, so the merge pass runs
+    its eight-threads-per-cell form (lists with 24 or more partial states); rows 5 per KV-head
+    group, the last page partial."""
+    w = synth.config2(3, batch=1, L=30000 - 7, layers=1)
+    w.n_q = np.array([5], dtype=np.int32)
+    q_bits, pool_bits, pool = _workload_case(w, 11)
+    ws = kap.Workspace(max_rows_per_item=5 * 4, max_batch=1)
+    got = gu.run_verify(q_bits, w.n_q, pool, w.bt_indptr, w.bt_pages, w.ctx_len, ws=ws)
+    info = ws.info()
+    assert info["n_items"] // 8 >= 24 and info["n_merge_groups"] == 8
+    ws.close()
+    _check_pair(got, gu.oracle_verify(q_bits, w.n_q, pool_bits, w.bt_indptr, w.bt_pages, w.ctx_len), "long verify")
+    # the proposal path over the identity plan, at most 8 pages per CTA: 235 states per list
+    w.force_full = np.ones(1, dtype=np.uint8)
+    plan = kap.compile_workload(w)
+    assert plan["plan_flags"][0] & kap.PLAN_FULL
+    qd = _decode_rows(w, q_bits)
+    _check_pair(gu.run_decode(qd, pool, plan, w.ctx_len, max_chunk_pages=8),
+                gu.oracle_decode(qd, pool_bits, plan, w.ctx_len), "long decode, 8 pages per CTA")
 
 
 @pytest.mark.parametrize("cluster", [1, 2, 5, 8, 13, 16])
