@@ -138,7 +138,8 @@ kap_status kap_compile_plan(
  *   max_rows_per_item  most query rows of one (sequence, KV head): n_q * (Hq / Hkv)
  *   max_batch          most sequences
  * kap_schedule (HOST arrays) splits every (sequence, KV head) page list of list_len[b] pages into
- * near-equal contiguous chunks so that the chunks fill the GPU in whole waves, uploads the work
+ * near-equal contiguous chunks so that the chunks fill the GPU in whole waves (short lists: a half
+ * or a quarter of one, so that a CTA has more than a page or two to stream), uploads the work
  * list on `cuda_stream` (asynchronous copy from pinned memory owned by the workspace) and keeps
  * it until the next kap_schedule.  The schedule depends only on the page counts, so one schedule
  * serves every layer and every step whose list lengths and row counts are unchanged; a call that
