@@ -118,3 +118,19 @@ def test_cluster_schedules():
                                                                max_items=100000, max_cluster=mc)
         assert 1 <= cluster <= mc
         _verify_schedule(n, nq, items, 8, PROPOSAL_CAP if nq is None else VERIFY_CAP, cluster)
+
+
+def test_short_lists_are_not_cut_into_single_pages():
+    """One 4K sequence (45 selected pages per KV head, 256 for verification): a CTA per page plus a
+    merge pass over dozens of partial states costs more than it spreads.  The candidates include
+    launches that fill a half or a quarter of a wave and the merge pass is charged per batch of 16
+    partial states, so the choice is a cluster per list (no merge pass) or a few pages per CTA."""
+    items, n_merge, max_chunk, cluster = kap.schedule_host([45], None, 32, 8, 444, max_cluster=16)
+    ctas = len(items) * cluster
+    assert ctas <= 148 and max_chunk >= 3
+    assert n_merge == 0 or max(items[:, 6]) <= 16
+    items, n_merge, max_chunk = kap.schedule_host([256], [4], 32, 8, 444)
+    assert len(items) <= 222 and max_chunk >= 8 and max(items[:, 6]) <= 32
+    # long lists still fill the wave
+    items, n_merge, max_chunk = kap.schedule_host([8192] * 4, [4] * 4, 32, 8, 444)
+    assert len(items) >= 432
