@@ -962,6 +962,8 @@ def main():
     ap.add_argument("--pdl", type=int, default=-1)
     ap.add_argument("--ctas-per-sm", type=int, default=-1)
     ap.add_argument("--early-kv", type=int, default=-1)
+    ap.add_argument("--verify-kernel", type=int, default=0, choices=[0, 1],
+                    help="kap_set_verify_kernel: 0 = mma.sync split kernel (default), 1 = tcgen05 kernel")
     ap.add_argument("--kv-layout", default="hnd", choices=["hnd", "nhd"],
                     help="pool layout given to the attention calls (default: head-major)")
     args = ap.parse_args()
@@ -990,6 +992,7 @@ def main():
     else:
         seed = 0
     kap.set_launch_options(args.pdl, args.early_kv, args.ctas_per_sm, args.max_cluster, args.ring_slots)
+    kap.set_verify_kernel(args.verify_kernel)
     solo = rank == 0 and world == 1
 
     res, cy = measure(args.config, args, dev, seed, group, world, layers=args.layers, want_extras=solo)
@@ -1003,7 +1006,7 @@ def main():
         "config": config_dict(w, k, cy.layers, {"parallelism": f"dp{world} (independent batches per GPU)",
                                                  "pdl": args.pdl, "max_cluster": args.max_cluster, "ring_slots": args.ring_slots,
                                                  "ctas_per_sm": args.ctas_per_sm, "early_kv": args.early_kv,
-                                                 "kv_layout": args.kv_layout}),
+                                                 "kv_layout": args.kv_layout, "verify_kernel": args.verify_kernel}),
         "clocks": res["clocks"], "per_step": res["per_step"], "e2e": res.get("e2e"),
         "gpu_launches": res["gpu_launches"],
         "roofline": res[dominant], "roofline_decode": res["decode"], "roofline_verify": res["verify"],
@@ -1033,6 +1036,23 @@ def main():
                 c2.free()
             except Exception as e:       # a side measurement must not lose the main line
                 also[name] = {"error": repr(e)}
+        try:       # verification through the tcgen05 kernel (8 layers each), for the record: it is the slower one
+            kap.set_verify_kernel(1)
+            tc = {}
+            for name in ("c4", "c3"):
+                c3 = Cycle(name, 0, layers=8, device=dev, kv_layout=args.kv_layout)
+                c3.capture()
+                _, _, _, st = c3.time_steps(3, 3, min_replays=20, min_seconds=0.3)
+                tc[name] = {"us_per_layer_verify_mean_median_best": [round(st["us_per_layer_verify"][q], 2) for q in ("mean", "median", "best")],
+                            "verify_frac_of_8TBs": round(c3.verify_bytes / (st["us_per_layer_verify"]["mean"] * 1e-6) / 8e12, 4),
+                            "schedule": c3.info_v}
+                c3.free()
+            tc["note"] = "kap_set_verify_kernel(1): tcgen05.mma, accumulators in tensor memory; 8 layers"
+            also["verify_tcgen05"] = tc
+        except Exception as e:
+            also["verify_tcgen05"] = {"error": repr(e)}
+        finally:
+            kap.set_verify_kernel(args.verify_kernel)
         try:       # the headline configuration once more, as two interleaved micro-batches (8 layers)
             also[args.config + "_two_microbatches"] = time_two_microbatches(args.config, args, dev, 8)
         except Exception as e:

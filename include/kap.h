@@ -616,6 +616,19 @@ kap_status kap_workspace_check(kap_workspace* ws, void* cuda_stream);
 kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, int32_t ctas_per_sm,
                                   int32_t max_cluster, int32_t ring_slots);
 
+/* Which kernel runs kap_verify_attn (Section 3.2 "Full-context verification"); takes effect at the
+ * next kap_schedule of a verification workspace, process-wide.
+ *   0 (default)  the split kernel: mma.sync tiles of 16 query rows per warp.
+ *   1            the tcgen05 kernel: one tcgen05.mma per four pages for all query rows of a KV head,
+ *                accumulators in tensor memory, at most 32 query rows per KV head (n_q * Hq / Hkv;
+ *                schedules with more rows use the split kernel), slices of at most 1024 pages per
+ *                CTA, a 12-slot ring and two CTAs per SM whatever kap_set_launch_options says, no
+ *                clusters.  Same results within the tolerance of the path; on the paper-shaped
+ *                workloads it is the slower of the two on B200 (it keeps a page longer in its ring
+ *                slot), which is why it is not the default.
+ * The paper has no counterpart.  Error: KAP_ERR_INVALID_ARG for any other value. */
+kap_status kap_set_verify_kernel(int32_t kernel);
+
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t kap_launch_count(void);
 

@@ -13,7 +13,7 @@
 #include <vector>
 
 #include "kap_internal.h"
-#include "kap_attn_kernel.cuh"
+#include "kap_attn_umma_kernel.cuh"
 
 namespace kap {
 
@@ -74,6 +74,7 @@ std::atomic<int> g_max_cluster{kMaxCluster};       // largest thread-block clust
 std::atomic<int> g_early_kv{1};
 std::atomic<int> g_ring_slots{kDefaultSlots};
 std::atomic<int> g_ctas_per_sm{0};       // 0 = as many as fit (occupancy)
+std::atomic<int> g_verify_kernel{0};     // verification launches: 0 = kap_attn_split_kernel (mma.sync), 1 = kap_attn_umma_kernel (tcgen05)
 constexpr int kWideMergeSplits = 24;     // partial states per list from which the wide merge kernel pays off ...
 constexpr int64_t kWideMergeRows = 1024; // ... as long as (lists x query rows) stays below this
 
@@ -192,6 +193,10 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
             cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             cudaGetLastError();
         }
+        for (const void* fn : {(const void*)kap_attn_umma_kernel<false>, (const void*)kap_attn_umma_kernel<true>}) {
+            cudaError_t ae = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, umma_smem_bytes());
+            if (ae != cudaSuccess) return fail(KAP_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ae));
+        }
         ws->attrs_set = 1;
     }
 
@@ -225,7 +230,7 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)ws->n_items * (unsigned)ws->cluster_size);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem_bytes_for(ws->ring_slots);
+    cfg.dynamicSmemBytes = ws->umma ? umma_smem_bytes() : smem_bytes_for(ws->ring_slots);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
@@ -237,7 +242,13 @@ kap_status launch_attention(const AttnParams& p_in, const void* pool, int64_t pa
     if (!plain && !push && ws->max_chunk > kMaxIds)
         return fail(KAP_ERR_INVALID_ARG, "the schedule's slices of %d pages need plain page lists (no logical "
                     "indices, no masks)", ws->max_chunk);
-    if (push && nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<1, true>, *map, p));
+    if (ws->umma) {
+        if (!plain || !p.q_indptr || ws->cluster_size != 1 || ws->ring_slots != kUmmaSlots)
+            return fail(KAP_ERR_INVALID_ARG, "the schedule was made for the tcgen05 verification kernel: plain page lists with q_indptr only");
+        if (nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_umma_kernel<true>, *map, p));
+        else KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_umma_kernel<false>, *map, p));
+    }
+    else if (push && nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<1, true>, *map, p));
     else if (push) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<1, false>, *map, p));
     else if (plain && nhd) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<2, true>, *map, p));
     else if (plain) KAP_CUDA(cudaLaunchKernelEx(&cfg, kap_attn_split_kernel<2, false>, *map, p));
@@ -359,6 +370,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     key.push_back(batch); key.push_back(num_q_heads); key.push_back(num_kv_heads);
     key.push_back(max_chunk_pages); key.push_back(n_q != nullptr);
     key.push_back(g_ring_slots.load()); key.push_back(g_ctas_per_sm.load()); key.push_back(g_max_cluster.load());
+    key.push_back(g_verify_kernel.load());
     for (int32_t b = 0; b < batch && list_len; ++b) { key.push_back(list_len[b]); key.push_back(n_q ? n_q[b] : 1); }
     if (ws->schedule_key && *ws->schedule_key == key) return KAP_OK;
     std::vector<WorkItem> items;
@@ -368,7 +380,10 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     // clusters of 2, 4, 8 CTAs fit a few less (GPC boundaries)
     DeviceScope scope(ws->device);                // the caller's current device is put back on return
     KAP_CUDA(scope.err);
-    const int ring_slots = g_ring_slots.load();
+    // the tcgen05 verification kernel: 32 query rows at most, a 12-slot ring, two CTAs per SM, no clusters
+    bool umma = n_q != nullptr && g_verify_kernel.load() == 1;
+    for (int32_t b = 0; umma && b < batch; ++b) umma = n_q[b] * (num_q_heads / std::max(num_kv_heads, 1)) <= kUmmaRows;
+    const int ring_slots = umma ? kUmmaSlots : g_ring_slots.load();
     if (!offsets_fit_ring(batch, n_q != nullptr, ring_slots))
         return fail(KAP_ERR_CAPACITY, "batch %d: the kernel stages the batch's offset arrays in its %d-slot ring "
                     "(%d bytes)", batch, ring_slots, ring_slots * kPageHeadBytes);
@@ -376,10 +391,18 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     cudaFuncSetAttribute(kap_attn_split_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          smem_bytes_for(kMaxSlots));
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel<0, false>, kThreads, smem) != cudaSuccess || occ < 1)
-        occ = 1;
+    cudaError_t oe;
+    if (umma) {
+        cudaFuncSetAttribute(kap_attn_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, umma_smem_bytes());
+        oe = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_umma_kernel<false>, kThreads, umma_smem_bytes());
+    } else {
+        oe = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kap_attn_split_kernel<0, false>, kThreads, smem);
+    }
+    if (oe != cudaSuccess || occ < 1) occ = 1;
     const int want = g_ctas_per_sm.load();
-    const int per_sm = want > 0 ? std::min(want, occ) : occ;
+    // (the occupancy query answers 1 for any kernel that allocates tensor memory; two CTAs of 110 KiB and 256
+    // columns each do become resident together - measured - so the schedule counts on two)
+    const int per_sm = umma ? 2 : want > 0 ? std::min(want, occ) : occ;
     // (nothing of the workspace changes until the new schedule is complete: a failure below leaves
     // the previous schedule, ring size and cluster size in force together)
     const int32_t ctas_per_wave = per_sm * ws->sm_count;
@@ -387,7 +410,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     cudaFuncSetAttribute(kap_attn_split_kernel<0, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     cudaGetLastError();
     for (int c = 2; c <= kMaxCluster; ++c) {
-        if (c > g_max_cluster.load()) continue;
+        if (c > g_max_cluster.load() || umma) { slots[c - 1] = 0; continue; }
         cudaLaunchAttribute ca[1];
         ca[0].id = cudaLaunchAttributeClusterDimension;
         ca[0].val.clusterDim.x = (unsigned)c; ca[0].val.clusterDim.y = 1; ca[0].val.clusterDim.z = 1;
@@ -410,7 +433,8 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
         one_wave[c - 1] = (int32_t)((int64_t)slots[c - 1] * keep / per_sm);
     int32_t cluster = 1;
     kap_status st = build_schedule(batch, list_len, n_q, num_q_heads, num_kv_heads, slots, one_wave,
-                                   max_chunk_pages, ws->max_items, ws->max_rows, items, groups,
+                                   umma ? (max_chunk_pages > 0 ? std::min(max_chunk_pages, kUmmaIds) : kUmmaIds) : max_chunk_pages,
+                                   ws->max_items, ws->max_rows, items, groups,
                                    &max_chunk, &row_tiles, &cluster);
     if (st != KAP_OK) return st;
     if ((int64_t)items.size() > ws->max_items || (int64_t)groups.size() > ws->max_items)
@@ -442,7 +466,7 @@ extern "C" kap_status kap_schedule(kap_workspace* ws, int32_t batch, const int32
     ws->batch = batch; ws->n_items = (int32_t)items.size(); ws->n_groups = (int32_t)groups.size();
     ws->n_merge_groups = n_merge; ws->max_chunk = max_chunk; ws->row_tiles = row_tiles;
     ws->num_q_heads = num_q_heads; ws->num_kv_heads = num_kv_heads; ws->has_nq = n_q != nullptr;
-    ws->total_rows = total_rows; ws->cluster_size = cluster; ws->max_splits = max_splits;
+    ws->total_rows = total_rows; ws->cluster_size = cluster; ws->umma = umma ? 1 : 0; ws->max_splits = max_splits;
     int32_t mq = 1;
     for (int32_t b = 0; b < batch; ++b) mq = std::max(mq, n_q ? n_q[b] : 1);
     ws->max_nq = mq;
@@ -535,6 +559,12 @@ extern "C" kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, 
     if (early_kv >= 0) g_early_kv.store(early_kv ? 1 : 0);
     if (ctas_per_sm >= 0) g_ctas_per_sm.store(ctas_per_sm);
     if (max_cluster > 0) g_max_cluster.store(max_cluster);
+    return KAP_OK;
+}
+
+extern "C" kap_status kap_set_verify_kernel(int32_t kernel) {
+    if (kernel != 0 && kernel != 1) return fail(KAP_ERR_INVALID_ARG, "kernel %d (0 = mma.sync, 1 = tcgen05)", kernel);
+    g_verify_kernel.store(kernel);
     return KAP_OK;
 }
 

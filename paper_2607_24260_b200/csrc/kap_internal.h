@@ -50,6 +50,7 @@ struct kap_workspace {
     // last schedule
     int32_t batch = 0, n_items = 0, n_groups = 0, n_merge_groups = 0, max_chunk = 0;
     int32_t max_splits = 1;                  // most partial states any list of the schedule has
+    int32_t umma = 0;                        // the schedule was made for kap_attn_umma_kernel (tcgen05)
     int32_t ctas_per_wave = 0, row_tiles = 1, num_q_heads = 0, num_kv_heads = 0;
     int32_t has_nq = 0;            // schedule was made with an n_q array (verification path)
     int32_t kv_layout = 0;         // KAP_KV_HND / KAP_KV_NHD: layout of the pools given to the attention calls

@@ -63,6 +63,7 @@ SIGNATURES = {
     "kap_device_sm_rates": (C.c_int, [C.c_int32, C.c_int32, _f32p, _i32p]),
     "kap_workspace_check": (C.c_int, [_vp, _vp]),
     "kap_set_launch_options": (C.c_int, [C.c_int32] * 5),
+    "kap_set_verify_kernel": (C.c_int, [C.c_int32]),
     "kap_launch_count": (C.c_int64, []),
     "kap_last_error": (C.c_char_p, []),
     "kap_version": (C.c_char_p, []),
@@ -117,6 +118,12 @@ def set_launch_options(use_pdl: int = -1, early_kv: int = -1, ctas_per_sm: int =
                        max_cluster: int = -1, ring_slots: int = -1):
     _check(lib().kap_set_launch_options(int(use_pdl), int(early_kv), int(ctas_per_sm),
                                         int(max_cluster), int(ring_slots)))
+
+
+def set_verify_kernel(kernel: int):
+    """kap_set_verify_kernel: 0 = the mma.sync split kernel, 1 = the tcgen05 kernel (schedules made
+    afterwards; at most 64 query rows per KV head, else the split kernel is used)."""
+    _check(lib().kap_set_verify_kernel(int(kernel)))
 
 
 # ------------------------------------------------------------------------------- kap_compile_plan
