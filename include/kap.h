@@ -624,8 +624,8 @@ kap_status kap_set_launch_options(int32_t use_pdl, int32_t early_kv, int32_t cta
  *                schedules with more rows use the split kernel), slices of at most 1024 pages per
  *                CTA, a 12-slot ring and two CTAs per SM whatever kap_set_launch_options says, no
  *                clusters.  Same results within the tolerance of the path; on the paper-shaped
- *                workloads it is the slower of the two on B200 (it keeps a page longer in its ring
- *                slot), which is why it is not the default.
+ *                workloads it is the slower of the two on B200 by 10-20 % (it keeps a page longer
+ *                in its ring slot), which is why it is not the default.
  * The paper has no counterpart.  Error: KAP_ERR_INVALID_ARG for any other value. */
 kap_status kap_set_verify_kernel(int32_t kernel);
 

@@ -5,18 +5,20 @@
 // once per row tile (ldmatrix + mma.sync); from two row tiles on (k = 8 drafts x 4 heads = 32 rows)
 // the SM's shared-memory and issue bandwidth, not HBM, set the pace.  Here one thread issues, per
 // batch of four pages,
-//     S = Q K^T     eight  tcgen05.mma  128 x 64 x 16   (A = the Q tile, B = the four K tiles, both
+//     S = Q K^T     eight  tcgen05.mma  64 x 64 x 16    (A = the Q tile, B = the four K tiles, both
 //                   in shared memory, K-major, 128-byte swizzle: K exactly as the TMA copies left it)
-//     O += P V      four   tcgen05.mma  128 x 128 x 16  (A = P from tensor memory, B = one V tile,
+//     O += P V      four   tcgen05.mma  64 x 128 x 16   (A = P from tensor memory, B = one V tile,
 //                   MN-major, same swizzle)
 // for all query rows at once: a tile is read from shared memory once, by the tensor core.  (A
 // tcgen05.mma of this shape costs about 48 cycles whether N is 16 or 64 - measured - so scores are
-// computed four pages at a time.)  Rows live in TMEM lanes (row r = lane r; 32 of the 128 are
-// used), one softmax thread per row reads its 64 scores with tcgen05.ld and writes its 64 weights
-// back as packed bf16 over the scores it has read.
+// computed four pages at a time.)  Rows live in TMEM lanes: with 64-row tiles row r is lane
+// (r % 16) + 32 (r / 16), i.e. rows 0-15 in the first 16 lanes of warp 0's quarter and rows 16-31 in
+// the first 16 lanes of warp 1's; one softmax thread per row reads its 64 scores with tcgen05.ld
+// and writes its 64 weights back as packed bf16 over the scores it has read.  (128-row tiles were
+// tried first: twice the tensor work for the same 32 rows, and under the power cap the slower.)
 //
 // Roles of the four warps:
-//   warp 0   softmax: one query row per thread
+//   warps 0, 1  softmax: one query row per thread, 16 rows per warp (warp 1 only with more than 16 rows)
 //   warp 2   lane 0 refills the shared-memory ring with TMA copies, a batch of four pages at a time
 //   warp 3   lane 0 issues the MMAs: S of batch g + 1 is issued before O += P V of batch g, so the
 //            tensor core computes the next scores while the softmax threads work on these
@@ -25,7 +27,7 @@
 // rescaled in tensor memory - after the previous batch's P V has completed and before this batch's is
 // issued.  out = sum(p v) / sum(p) with the same rounded p in both sums, as in the other kernel.
 //
-// Shared memory: control block (page ids, barriers) 8 KiB, Q tile 8 KiB (32 rows; the MMA reads 128
+// Shared memory: control block (page ids, barriers) 6 KiB, Q tile 8 KiB (32 rows; the MMA reads 64
 // rows from there on, i.e. on into the ring - those rows' results are never looked at), ring of 12
 // pages as four planes (K columns 0-63, K columns 64-127, V likewise) so that the K tiles of a batch
 // are one contiguous 64-row operand.  Tensor memory: 256 columns per CTA (two S / P buffers of 64,
@@ -141,7 +143,8 @@ kap_attn_umma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParam
         offs[p.batch + 1 + t] = p.q_indptr[t];
     }
     __syncthreads();
-    const int rows = item.n_q * p.G;                         // <= 32: row r lives in TMEM lane r
+    const int rows = item.n_q * p.G;                         // <= 32; row r lives in TMEM lane (r % 16) + 32 (r / 16)
+    const int n_soft = rows > 16 ? 2 : 1;                    // softmax warps: 16 rows each (lanes 0-15 of the warp's TMEM quarter)
     int n_local = item.page_end - item.page_begin;
     if (n_local > kUmmaIds) {                                // the scheduler caps this kernel's slices at 1024 pages
         if (tid == 0) atomicOr(p.status, 1 << KAP_ERR_DEVICE_INDEX);
@@ -162,7 +165,7 @@ kap_attn_umma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParam
         for (int g = 0; g < n_slots / kUmmaBatch; ++g) mbar_init(smem_u32(&ub->batch_free[g]), 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ub->s_ready[b]), 1);
-            mbar_init(smem_u32(&ub->p_ready[b]), 1);
+            mbar_init(smem_u32(&ub->p_ready[b]), (uint32_t)n_soft);
             mbar_init(smem_u32(&ub->o_done[b]), 1);
         }
         tail->timed_out = 0;
@@ -238,7 +241,7 @@ kap_attn_umma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParam
         }
     } else if (warp == 3 && lane == 0) {
         // ---- tensor core: S of batch g, then O += P V of batch g - 1
-        constexpr uint32_t idesc_s = umma_idesc(128, kUmmaBatch * kPageSize, false), idesc_o = umma_idesc(128, kHeadDim, true);
+        constexpr uint32_t idesc_s = umma_idesc(64, kUmmaBatch * kPageSize, false), idesc_o = umma_idesc(64, kHeadDim, true);
         auto issue_pv = [&](int g) {                         // false: a wait ran out
             const int b = g & 1;
             if (!mbar_wait(smem_u32(&ub->p_ready[b]), (uint32_t)(g >> 1) & 1u, deadline, &tail->timed_out)) return false;
@@ -265,7 +268,7 @@ kap_attn_umma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParam
             if (ok && g >= 2) ok = mbar_wait(smem_u32(&ub->o_done[b]), (uint32_t)((g - 2) >> 1) & 1u, deadline, &tail->timed_out);
             if (!ok) break;
             tc_fence_after();
-            // Q: 128 rows (M) x 128 columns (K); K: the batch's 64 token rows (N); 16 columns per MMA, 8 rows = 1 KiB
+            // Q: 64 rows (M) x 128 columns (K); K: the batch's 64 token rows (N); 16 columns per MMA, 8 rows = 1 KiB
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const uint32_t q_at = smem_u32(q_tile + (ks >> 2) * (kUmmaQBytes / 2) + (ks & 3) * 32);
@@ -276,10 +279,10 @@ kap_attn_umma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParam
             if (g > 0) ok = issue_pv(g - 1);
         }
         if (ok) issue_pv(n_batches - 1);
-    } else if (warp == 0) {
-        // ---- softmax: one query row per thread, a batch of 64 scores at a time
-        const int R = lane;
-        const bool valid = R < rows;
+    } else if (warp < n_soft) {
+        // ---- softmax: one query row per thread (16 per warp), a batch of 64 scores at a time
+        const int R = warp * 16 + lane;
+        const bool valid = lane < 16 && R < rows;
         const int pos = L - item.n_q + (valid ? R / p.G : item.n_q - 1);   // this row's logical position
         const int full_vis_limit = L - item.n_q;
         const float sc = p.scale_log2;
@@ -312,7 +315,7 @@ kap_attn_umma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParam
                 // value rows past the context's end may hold anything (even NaN): zero them
                 for (int pg = 0; pg < cnt; ++pg) {
                     const int first_bad = L - (tok0 + pg * kPageSize);
-                    if (first_bad < kPageSize) {
+                    if (first_bad < kPageSize && warp == 0) {
                         unsigned char* v_tile = ring + 2 * kUmmaPlaneBytes + ((g * kUmmaBatch + pg) % n_slots) * kHalfTileBytes;
                         if (lane < 16)
                             for (int r = max(first_bad, 0); r < kPageSize; ++r)
